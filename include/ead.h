@@ -1,0 +1,163 @@
+/*
+ * ead.h - C ABI of the B200 (sm_100a) library for the gate step of Entropy
+ * Adaptive Decoding (EAD).
+ *
+ * One "gate step" is one pass through the loop body of the paper's
+ * Algorithm 1 for a batch of B independent sequences: project the active
+ * model's final hidden state through that model's LM head (the last stage of
+ * "l <- M_t(x + y)"), take the softmax of the raw logits (Eq. 1) and its
+ * Shannon entropy (Eq. 2), pick the greedy token (the temperature -> 0 limit
+ * of the sampling lines), append the entropy to the sequence's window and
+ * average the last w entries (Eq. 3 / "mean(W[-w:])"), count the token
+ * (c <- c + 1) and apply the dwell + threshold rule (Eq. 4) that selects the
+ * model for the next token.
+ *
+ * Conventions
+ *   - Every function returns 0 (EAD_OK) or a negative EAD_E* code; nothing
+ *     throws or aborts across this boundary.  ead_strerror names a code.
+ *   - Pointers marked "dev" are device pointers on cfg.device, "host" are
+ *     host pointers.  Weights, hidden states and outputs are BORROWED: the
+ *     library never copies or frees them; they must stay valid until the work
+ *     enqueued with them has finished.  All per-sequence state (window,
+ *     dwell counter, model flag) is OWNED by the context.
+ *   - bf16 matrices are row major; their base must be 16-byte aligned and
+ *     H_small, H_large must be multiples of 8 (16-byte rows).
+ *   - Work is enqueued on cfg.stream and is asynchronous with respect to the
+ *     host unless stated otherwise.  Calls on one context must not overlap on
+ *     the device (one stream); the context is not thread safe.
+ *   - The library needs an sm_100 device and has no other code path:
+ *     ead_create fails with EAD_EUNSUPPORTED_ARCH elsewhere.
+ *   - Models are numbered 0 = small (M_S), 1 = large (M_L).
+ */
+#ifndef EAD_H_
+#define EAD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define EAD_OK                  0
+#define EAD_EINVALID_ARG      (-1)  /* NULL where not allowed, size out of range            */
+#define EAD_EALIGNMENT        (-2)  /* pointer not 16-byte aligned or H not a multiple of 8 */
+#define EAD_ECUDA             (-3)  /* a CUDA runtime / driver call failed                  */
+#define EAD_EUNSUPPORTED_ARCH (-4)  /* device is not sm_100                                 */
+#define EAD_EDEVICE_FAULT     (-5)  /* the device status word reports a kernel-side error   */
+#define EAD_ESTATE            (-6)  /* state blob of the wrong size or version              */
+
+/* Bits of the device status word (ead_status). */
+#define EAD_STATUS_NONFINITE   0x1u /* some row saw a NaN / infinite logit (row gets H = NaN) */
+#define EAD_STATUS_WAIT_EXPIRED 0x2u /* a bounded wait inside a kernel ran out                 */
+#define EAD_STATUS_BAD_COUNT   0x4u /* internal row counts inconsistent                       */
+
+typedef struct ead_ctx ead_ctx; /* opaque */
+
+/* Hyper-parameters follow the "Require" line of Algorithm 1 (tau, w, d_min);
+ * the paper's experiments use w = 5 and d_min = 10. */
+typedef struct ead_config {
+    int32_t B;           /* sequences in the batch, 1 .. 4096                                 */
+    int32_t V;           /* vocabulary size shared by both heads, >= 1                        */
+    int32_t H_small;     /* hidden size of M_S, multiple of 8, >= 8                           */
+    int32_t H_large;     /* hidden size of M_L, multiple of 8, >= 8                           */
+    int32_t w;           /* window length of Eq. 3, 1 .. 64                                   */
+    int32_t d_min;       /* minimum tokens on a model before a switch (Eq. 4); <= 1 = none    */
+    float   tau;         /* threshold of Eq. 4, compared with the rolling mean in `unit`      */
+    int32_t unit;        /* 0: entropy in nats; 1: in bits (Eq. 2 as printed, log base 2)     */
+    int32_t start_model; /* model of the first token; Algorithm 1 starts on 0 (small)         */
+    int32_t device;      /* CUDA device ordinal                                               */
+    void   *stream;      /* cudaStream_t to enqueue on (borrowed); NULL = legacy default      */
+} ead_config;
+
+/*
+ * Creates a context: allocates the per-sequence state of Algorithm 1's
+ * initialisation (empty window, c = 0, M_t = start_model) plus scratch, and
+ * encodes the TMA descriptors of the two heads.
+ *   W_small  dev, bf16 [V, H_small], one row per vocabulary entry (borrowed, read only)
+ *   W_large  dev, bf16 [V, H_large]
+ *   out      host, receives the context
+ * Synchronises the device once.  Errors: EAD_EINVALID_ARG, EAD_EALIGNMENT,
+ * EAD_EUNSUPPORTED_ARCH, EAD_ECUDA.
+ */
+int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, ead_ctx **out);
+
+/*
+ * One gate step (one iteration of Algorithm 1's loop) for all B sequences.
+ *   h_small     dev, bf16 [B, H_small]: final hidden state of M_S per sequence
+ *   h_large     dev, bf16 [B, H_large]: the same for M_L
+ *               Only the row of the model that is active for a sequence is read.
+ *   tok         dev, int32 [B]: greedy token (lowest index among equal maxima; -1 for a
+ *               row with non-finite logits)
+ *   H           dev, float [B]: entropy of Eq. 2 in cfg.unit
+ *   Hbar        dev, float [B]: rolling mean of Eq. 3 after this token
+ *   model_used  dev, uint8 [B]: model that produced this token
+ *   next_model  dev, uint8 [B]: model selected for the next token (Eq. 4)
+ * Any output pointer may be NULL to skip it.  Row b of every output belongs to
+ * row b of the inputs.  Asynchronous.  Errors: EAD_EINVALID_ARG,
+ * EAD_EALIGNMENT, EAD_ECUDA.
+ */
+int ead_step(ead_ctx *ctx, const void *h_small, const void *h_large, int32_t *tok, float *H,
+             float *Hbar, uint8_t *model_used, uint8_t *next_model);
+
+/*
+ * T consecutive gate steps with the hidden states of all steps resident on
+ * the device; step t reads h_*_seq[t] and writes row t of each output.  The
+ * T-step loop is replayed from CUDA graphs; the result is bit-identical to T
+ * calls of ead_step.  Continues from the context's current state.
+ *   h_small_seq  dev, bf16 [T, B, H_small];  h_large_seq  dev, bf16 [T, B, H_large]
+ *   outputs      dev, [T, B] each, as in ead_step; any may be NULL
+ * Asynchronous.  Errors as ead_step.
+ */
+int ead_run(ead_ctx *ctx, int32_t T, const void *h_small_seq, const void *h_large_seq,
+            int32_t *tok, float *H, float *Hbar, uint8_t *model_used, uint8_t *next_model);
+
+/*
+ * The same T steps as ead_run, but every buffer is a HOST pointer: hidden
+ * states are copied to the device and results back through internal staging
+ * buffers, in chunks that overlap with the computation.  Synchronous: returns
+ * when the outputs are complete.  Any output may be NULL.  Pinned host memory
+ * makes the copies faster but is not required.
+ */
+int ead_run_host(ead_ctx *ctx, int32_t T, const void *h_small_seq, const void *h_large_seq,
+                 int32_t *tok, float *H, float *Hbar, uint8_t *model_used, uint8_t *next_model);
+
+/* Back to Algorithm 1's initial state (empty window, c = 0, start model) and a
+ * cleared status word.  Asynchronous. */
+int ead_reset(ead_ctx *ctx);
+
+/* Waits for the context's stream, then reports the device status word
+ * (EAD_STATUS_* bits, sticky until ead_reset).  Returns EAD_EDEVICE_FAULT if
+ * EAD_STATUS_WAIT_EXPIRED or EAD_STATUS_BAD_COUNT is set, else EAD_OK. */
+int ead_status(ead_ctx *ctx, uint32_t *status_word);
+
+/*
+ * Checkpoint of the per-sequence state (window contents, dwell counters, model
+ * flags, number of steps taken).  ead_state_size gives the blob size for this
+ * context; ead_get_state copies device -> host, ead_set_state host -> device.
+ * Both wait for the stream.  A blob is only valid for a context with the same
+ * B and w.  Errors: EAD_EINVALID_ARG, EAD_ESTATE, EAD_ECUDA.
+ */
+size_t ead_state_size(const ead_ctx *ctx);
+int ead_get_state(ead_ctx *ctx, void *host_blob, size_t size);
+int ead_set_state(ead_ctx *ctx, const void *host_blob, size_t size);
+
+/* Number of kernels the library has launched through this context so far
+ * (graph replays count their kernel nodes). */
+int64_t ead_kernel_launches(const ead_ctx *ctx);
+
+/* Launch geometry chosen at creation, for reporting: fills up to n ints with
+ * {CTAs of the LM-head kernel, pipeline stages, rows of the hidden-state TMA
+ * box, dynamic shared memory bytes}. */
+int ead_launch_info(const ead_ctx *ctx, int32_t *info, int32_t n);
+
+/* Waits for outstanding work and frees everything the context owns.  NULL is allowed. */
+void ead_destroy(ead_ctx *ctx);
+
+/* Static, NUL-terminated description of an EAD_E* code. */
+const char *ead_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EAD_H_ */

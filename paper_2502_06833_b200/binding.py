@@ -1,0 +1,174 @@
+"""ctypes binding of ``include/ead.h``: same names, argument marshalling only.
+
+PyTorch is used by callers for device memory and streams; every step of the
+gate path runs inside the CUDA library.  Tensors are passed as raw device
+pointers (``tensor.data_ptr()``), bf16 matrices as ``torch.bfloat16``.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_DIR, "libead_b200.so")
+
+EAD_OK = 0
+EAD_EINVALID_ARG = -1
+EAD_EALIGNMENT = -2
+EAD_ECUDA = -3
+EAD_EUNSUPPORTED_ARCH = -4
+EAD_EDEVICE_FAULT = -5
+EAD_ESTATE = -6
+EAD_STATUS_NONFINITE = 0x1
+EAD_STATUS_WAIT_EXPIRED = 0x2
+EAD_STATUS_BAD_COUNT = 0x4
+
+SYMBOLS = ["ead_create", "ead_step", "ead_run", "ead_run_host", "ead_reset", "ead_status",
+           "ead_state_size", "ead_get_state", "ead_set_state", "ead_kernel_launches",
+           "ead_launch_info", "ead_destroy", "ead_strerror"]
+
+
+class EadConfig(C.Structure):
+    _fields_ = [("B", C.c_int32), ("V", C.c_int32), ("H_small", C.c_int32), ("H_large", C.c_int32),
+                ("w", C.c_int32), ("d_min", C.c_int32), ("tau", C.c_float), ("unit", C.c_int32),
+                ("start_model", C.c_int32), ("device", C.c_int32), ("stream", C.c_void_p)]
+
+
+class EadError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads the CUDA library; fails loudly when it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2502_06833_b200.build` "
+                              "(there is no fallback path)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32p, f32p, u8p = C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p
+        L.ead_create.restype = C.c_int
+        L.ead_create.argtypes = [C.POINTER(EadConfig), vp, vp, C.POINTER(C.c_void_p)]
+        L.ead_step.restype = C.c_int
+        L.ead_step.argtypes = [vp, vp, vp, i32p, f32p, f32p, u8p, u8p]
+        for name in ("ead_run", "ead_run_host"):
+            f = getattr(L, name)
+            f.restype = C.c_int
+            f.argtypes = [vp, C.c_int32, vp, vp, i32p, f32p, f32p, u8p, u8p]
+        L.ead_reset.restype = C.c_int
+        L.ead_reset.argtypes = [vp]
+        L.ead_status.restype = C.c_int
+        L.ead_status.argtypes = [vp, C.POINTER(C.c_uint32)]
+        L.ead_state_size.restype = C.c_size_t
+        L.ead_state_size.argtypes = [vp]
+        L.ead_get_state.restype = C.c_int
+        L.ead_get_state.argtypes = [vp, vp, C.c_size_t]
+        L.ead_set_state.restype = C.c_int
+        L.ead_set_state.argtypes = [vp, vp, C.c_size_t]
+        L.ead_kernel_launches.restype = C.c_int64
+        L.ead_kernel_launches.argtypes = [vp]
+        L.ead_launch_info.restype = C.c_int
+        L.ead_launch_info.argtypes = [vp, C.POINTER(C.c_int32), C.c_int32]
+        L.ead_destroy.restype = None
+        L.ead_destroy.argtypes = [vp]
+        L.ead_strerror.restype = C.c_char_p
+        L.ead_strerror.argtypes = [C.c_int]
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().ead_strerror(int(code)).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != EAD_OK:
+        raise EadError(code, where)
+
+
+def _ptr(t):
+    """Device (or host) address of a torch tensor / numpy array / int / None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if hasattr(t, "data_ptr"):
+        return t.data_ptr()
+    return t.ctypes.data
+
+
+def ead_create(*, B, V, H_small, H_large, w, d_min, tau, W_small, W_large, unit=0, start_model=0,
+               device=0, stream=0):
+    """Returns an opaque context handle (int).  ``W_*`` are device bf16 ``[V, H]``; they are
+    borrowed, keep them alive until ``ead_destroy``."""
+    cfg = EadConfig(B, V, H_small, H_large, w, d_min, float(tau), unit, start_model, device,
+                    C.c_void_p(int(stream)))
+    out = C.c_void_p()
+    _check(lib().ead_create(C.byref(cfg), _ptr(W_small), _ptr(W_large), C.byref(out)), "ead_create")
+    return out.value
+
+
+def ead_step(ctx, h_small, h_large, tok=None, H=None, Hbar=None, model_used=None, next_model=None):
+    _check(lib().ead_step(ctx, _ptr(h_small), _ptr(h_large), _ptr(tok), _ptr(H), _ptr(Hbar),
+                          _ptr(model_used), _ptr(next_model)), "ead_step")
+
+
+def ead_run(ctx, T, h_small_seq, h_large_seq, tok=None, H=None, Hbar=None, model_used=None,
+            next_model=None):
+    _check(lib().ead_run(ctx, int(T), _ptr(h_small_seq), _ptr(h_large_seq), _ptr(tok), _ptr(H),
+                         _ptr(Hbar), _ptr(model_used), _ptr(next_model)), "ead_run")
+
+
+def ead_run_host(ctx, T, h_small_seq, h_large_seq, tok=None, H=None, Hbar=None, model_used=None,
+                 next_model=None):
+    """All buffers are HOST memory (numpy arrays or CPU tensors, ideally pinned)."""
+    _check(lib().ead_run_host(ctx, int(T), _ptr(h_small_seq), _ptr(h_large_seq), _ptr(tok), _ptr(H),
+                              _ptr(Hbar), _ptr(model_used), _ptr(next_model)), "ead_run_host")
+
+
+def ead_reset(ctx):
+    _check(lib().ead_reset(ctx), "ead_reset")
+
+
+def ead_status(ctx, raise_on_fault: bool = True) -> int:
+    word = C.c_uint32()
+    rc = lib().ead_status(ctx, C.byref(word))
+    if rc != EAD_OK and (raise_on_fault or rc != EAD_EDEVICE_FAULT):
+        raise EadError(rc, f"ead_status (status word {word.value:#x})")
+    return int(word.value)
+
+
+def ead_state_size(ctx) -> int:
+    return int(lib().ead_state_size(ctx))
+
+
+def ead_get_state(ctx) -> bytes:
+    n = ead_state_size(ctx)
+    buf = C.create_string_buffer(n)
+    _check(lib().ead_get_state(ctx, C.cast(buf, C.c_void_p), n), "ead_get_state")
+    return buf.raw
+
+
+def ead_set_state(ctx, blob: bytes) -> None:
+    buf = C.create_string_buffer(bytes(blob), len(blob))
+    _check(lib().ead_set_state(ctx, C.cast(buf, C.c_void_p), len(blob)), "ead_set_state")
+
+
+def ead_kernel_launches(ctx) -> int:
+    return int(lib().ead_kernel_launches(ctx))
+
+
+def ead_launch_info(ctx) -> dict:
+    a = (C.c_int32 * 4)()
+    _check(lib().ead_launch_info(ctx, a, 4), "ead_launch_info")
+    return dict(ctas=a[0], stages=a[1], a_rows=a[2], smem_bytes=a[3])
+
+
+def ead_destroy(ctx) -> None:
+    if ctx:
+        lib().ead_destroy(ctx)

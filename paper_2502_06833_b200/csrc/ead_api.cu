@@ -1,0 +1,545 @@
+// Host side of the C ABI declared in include/ead.h: context set-up (state, scratch,
+// TMA descriptors), step orchestration and CUDA-graph replay of the T-step loop.
+#include "../../include/ead.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "ead_internal.cuh"
+#include "gate_kernels.cuh"
+#include "lmhead_kernel.cuh"
+
+using namespace ead;
+
+namespace {
+
+constexpr int kGraphChunk = 32;           // gate steps unrolled in the replayed graph
+constexpr uint32_t kStateMagic = 0x45414431u;   // "EAD1"
+constexpr size_t kHostStageBytes = 64u << 20;   // per staging buffer of ead_run_host
+
+struct StateHeader {
+    uint32_t magic;
+    int32_t B, w, step;
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 matrix [rows, cols] row major -> tiles of box_rows x 64 elements, 128-byte swizzle,
+// out-of-range elements read as zero.
+bool encode_bf16_2d(CUtensorMap *tm, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {static_cast<cuuint32_t>(kBlockK), box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+struct ead_ctx {
+    ead_config cfg{};
+    cudaStream_t stream = nullptr;
+    cudaStream_t cap_stream = nullptr;     // capture happens on a private stream
+    int G = 0, a_rows = 0, stages = 0, slots_stride = 0;
+    size_t smem_bytes = 0;
+    const void *W[2] = {nullptr, nullptr};
+    // device state and scratch (owned)
+    StepCtl *ctl = nullptr;
+    RunArgs *args = nullptr;
+    uint8_t *flag = nullptr;
+    int32_t *c = nullptr, *nfill = nullptr, *perm = nullptr, *part_i = nullptr;
+    float *ring = nullptr, *part_m = nullptr, *part_s = nullptr, *part_t = nullptr;
+    uint16_t *hc[2] = {nullptr, nullptr};
+    CUtensorMap tmA[2], tmW[2], tmT[2];
+    cudaGraphExec_t g_one = nullptr, g_chunk = nullptr;
+    int64_t launches = 0;
+    // staging of ead_run_host (allocated on first use)
+    cudaStream_t in_stream = nullptr, out_stream = nullptr;
+    uint16_t *st_h[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};
+    void *st_out[2] = {nullptr, nullptr};
+    cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_comp[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
+    int st_steps = 0;
+};
+
+namespace {
+
+#define EAD_CUDA(x)                          \
+    do {                                     \
+        if ((x) != cudaSuccess) {            \
+            cudaGetLastError();              \
+            return EAD_ECUDA;                \
+        }                                    \
+    } while (0)
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// The three kernels of one gate step, in stream order.
+int enqueue_step(ead_ctx *x, cudaStream_t s)
+{
+    const ead_config &c = x->cfg;
+    const int cgrid = std::min(c.B, 4 * x->G);
+    ead_compact_kernel<<<cgrid, kCompactThreads, static_cast<size_t>(c.B) * sizeof(int32_t), s>>>(
+        x->ctl, x->args, x->flag, c.B, c.H_small, c.H_large, x->hc[0], x->hc[1], x->perm);
+
+    LmheadParams lp{};
+    lp.V = c.V;
+    lp.H[0] = c.H_small;
+    lp.H[1] = c.H_large;
+    lp.a_rows = x->a_rows;
+    lp.stages = x->stages;
+    lp.slots_stride = x->slots_stride;
+    lp.B = c.B;
+    lp.ctl = x->ctl;
+    lp.ctl_rw = x->ctl;
+    lp.part_m = x->part_m;
+    lp.part_s = x->part_s;
+    lp.part_t = x->part_t;
+    lp.part_i = x->part_i;
+    ead_lmhead_kernel<<<x->G, kLmheadThreads, x->smem_bytes, s>>>(x->tmA[0], x->tmA[1], x->tmW[0], x->tmW[1],
+                                                                  x->tmT[0], x->tmT[1], lp);
+
+    GateParams gp{};
+    gp.B = c.B;
+    gp.V = c.V;
+    gp.w = c.w;
+    gp.d_min = c.d_min;
+    gp.unit = c.unit;
+    gp.G = x->G;
+    gp.slots_stride = x->slots_stride;
+    gp.tau = c.tau;
+    gp.ctl = x->ctl;
+    gp.args = x->args;
+    gp.part_m = x->part_m;
+    gp.part_s = x->part_s;
+    gp.part_t = x->part_t;
+    gp.part_i = x->part_i;
+    gp.perm = x->perm;
+    gp.flag = x->flag;
+    gp.c = x->c;
+    gp.nfill = x->nfill;
+    gp.ring = x->ring;
+    const int rows_per_block = kGateThreads / 32;
+    ead_merge_gate_kernel<<<(c.B + rows_per_block - 1) / rows_per_block, kGateThreads, 0, s>>>(gp);
+    return cudaGetLastError() == cudaSuccess ? EAD_OK : EAD_ECUDA;
+}
+
+int build_graph(ead_ctx *x, int steps, cudaGraphExec_t *out)
+{
+    cudaGraph_t graph = nullptr;
+    EAD_CUDA(cudaStreamBeginCapture(x->cap_stream, cudaStreamCaptureModeThreadLocal));
+    int rc = EAD_OK;
+    for (int i = 0; i < steps && rc == EAD_OK; ++i) rc = enqueue_step(x, x->cap_stream);
+    cudaError_t e = cudaStreamEndCapture(x->cap_stream, &graph);
+    if (rc != EAD_OK || e != cudaSuccess || !graph) {
+        if (graph) cudaGraphDestroy(graph);
+        cudaGetLastError();
+        return EAD_ECUDA;
+    }
+    e = cudaGraphInstantiate(out, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return EAD_ECUDA;
+    }
+    return EAD_OK;
+}
+
+int set_args(ead_ctx *x, const void *hs, const void *hl, int32_t *tok, float *H, float *Hbar, uint8_t *used,
+             uint8_t *next, cudaStream_t s)
+{
+    RunArgs a{};
+    a.h[0] = static_cast<const uint16_t *>(hs);
+    a.h[1] = static_cast<const uint16_t *>(hl);
+    a.tok = tok;
+    a.H = H;
+    a.Hbar = Hbar;
+    a.used = used;
+    a.next = next;
+    ead_set_args_kernel<<<1, 32, 0, s>>>(x->args, a, x->ctl);
+    x->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? EAD_OK : EAD_ECUDA;
+}
+
+int run_device(ead_ctx *x, int T, const void *hs, const void *hl, int32_t *tok, float *H, float *Hbar,
+               uint8_t *used, uint8_t *next)
+{
+    int rc = set_args(x, hs, hl, tok, H, Hbar, used, next, x->stream);
+    if (rc != EAD_OK) return rc;
+    int left = T;
+    while (left >= kGraphChunk) {
+        EAD_CUDA(cudaGraphLaunch(x->g_chunk, x->stream));
+        left -= kGraphChunk;
+    }
+    while (left > 0) {
+        EAD_CUDA(cudaGraphLaunch(x->g_one, x->stream));
+        left -= 1;
+    }
+    x->launches += 3ll * T;
+    return EAD_OK;
+}
+
+void free_staging(ead_ctx *x)
+{
+    for (int i = 0; i < 2; ++i) {
+        for (int m = 0; m < 2; ++m) {
+            if (x->st_h[i][m]) cudaFree(x->st_h[i][m]);
+            x->st_h[i][m] = nullptr;
+        }
+        if (x->st_out[i]) cudaFree(x->st_out[i]);
+        x->st_out[i] = nullptr;
+        if (x->ev_in[i]) cudaEventDestroy(x->ev_in[i]);
+        if (x->ev_comp[i]) cudaEventDestroy(x->ev_comp[i]);
+        if (x->ev_out[i]) cudaEventDestroy(x->ev_out[i]);
+        x->ev_in[i] = x->ev_comp[i] = x->ev_out[i] = nullptr;
+    }
+    if (x->in_stream) cudaStreamDestroy(x->in_stream);
+    if (x->out_stream) cudaStreamDestroy(x->out_stream);
+    x->in_stream = x->out_stream = nullptr;
+    x->st_steps = 0;
+}
+
+// Bytes of one step of outputs in the staging layout: tok | H | Hbar | used | next,
+// each [steps, B], sections 16-byte aligned for a given number of steps.
+struct OutLayout {
+    size_t off_tok, off_H, off_Hbar, off_used, off_next, total;
+};
+OutLayout out_layout(int steps, int B)
+{
+    auto up = [](size_t v) { return (v + 255) & ~static_cast<size_t>(255); };
+    OutLayout l;
+    const size_t n = static_cast<size_t>(steps) * B;
+    l.off_tok = 0;
+    l.off_H = up(l.off_tok + 4 * n);
+    l.off_Hbar = up(l.off_H + 4 * n);
+    l.off_used = up(l.off_Hbar + 4 * n);
+    l.off_next = up(l.off_used + n);
+    l.total = up(l.off_next + n);
+    return l;
+}
+
+int ensure_staging(ead_ctx *x)
+{
+    if (x->st_steps) return EAD_OK;
+    const ead_config &c = x->cfg;
+    const size_t per_step = static_cast<size_t>(c.B) * (c.H_small + c.H_large) * 2;
+    int steps = static_cast<int>(std::max<size_t>(1, kHostStageBytes / per_step));
+    steps = std::min(steps, 256);
+    if (steps > kGraphChunk) steps -= steps % kGraphChunk;
+    EAD_CUDA(cudaStreamCreateWithFlags(&x->in_stream, cudaStreamNonBlocking));
+    EAD_CUDA(cudaStreamCreateWithFlags(&x->out_stream, cudaStreamNonBlocking));
+    const OutLayout l = out_layout(steps, c.B);
+    for (int i = 0; i < 2; ++i) {
+        EAD_CUDA(cudaMalloc(&x->st_h[i][0], static_cast<size_t>(steps) * c.B * c.H_small * 2));
+        EAD_CUDA(cudaMalloc(&x->st_h[i][1], static_cast<size_t>(steps) * c.B * c.H_large * 2));
+        EAD_CUDA(cudaMalloc(&x->st_out[i], l.total));
+        EAD_CUDA(cudaEventCreateWithFlags(&x->ev_in[i], cudaEventDisableTiming));
+        EAD_CUDA(cudaEventCreateWithFlags(&x->ev_comp[i], cudaEventDisableTiming));
+        EAD_CUDA(cudaEventCreateWithFlags(&x->ev_out[i], cudaEventDisableTiming));
+    }
+    x->st_steps = steps;
+    return EAD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *ead_strerror(int code)
+{
+    switch (code) {
+        case EAD_OK: return "ok";
+        case EAD_EINVALID_ARG: return "invalid argument";
+        case EAD_EALIGNMENT: return "pointer not 16-byte aligned or hidden size not a multiple of 8";
+        case EAD_ECUDA: return "CUDA call failed";
+        case EAD_EUNSUPPORTED_ARCH: return "device is not sm_100";
+        case EAD_EDEVICE_FAULT: return "device status word reports a kernel-side error";
+        case EAD_ESTATE: return "state blob does not match this context";
+        default: return "unknown error";
+    }
+}
+
+int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, ead_ctx **out)
+{
+    if (!cfg || !W_small || !W_large || !out) return EAD_EINVALID_ARG;
+    *out = nullptr;
+    if (cfg->B < 1 || cfg->B > 4096 || cfg->V < 1 || cfg->H_small < 8 || cfg->H_large < 8 || cfg->w < 1 ||
+        cfg->w > 64 || (cfg->unit != 0 && cfg->unit != 1) || (cfg->start_model != 0 && cfg->start_model != 1))
+        return EAD_EINVALID_ARG;
+    if (cfg->H_small % 8 || cfg->H_large % 8 || !aligned16(W_small) || !aligned16(W_large)) return EAD_EALIGNMENT;
+
+    int ndev = 0;
+    EAD_CUDA(cudaGetDeviceCount(&ndev));
+    if (cfg->device < 0 || cfg->device >= ndev) return EAD_EINVALID_ARG;
+    EAD_CUDA(cudaSetDevice(cfg->device));
+    cudaDeviceProp prop;
+    EAD_CUDA(cudaGetDeviceProperties(&prop, cfg->device));
+    if (prop.major != 10) return EAD_EUNSUPPORTED_ARCH;
+
+    ead_ctx *x = new (std::nothrow) ead_ctx();
+    if (!x) return EAD_ECUDA;
+    x->cfg = *cfg;
+    x->stream = static_cast<cudaStream_t>(cfg->stream);
+    x->W[0] = W_small;
+    x->W[1] = W_large;
+    x->G = prop.multiProcessorCount;
+    x->slots_stride = (x->G + 31) & ~31;
+    x->a_rows = std::min(kTileM, (cfg->B + 7) & ~7);
+    const size_t stage_bytes = static_cast<size_t>(x->a_rows) * kBlockK * 2 + kWTileBytes;
+    const size_t smem_max = prop.sharedMemPerBlockOptin;
+    x->stages = static_cast<int>(std::min<size_t>(kMaxStages, (smem_max - kSmemCtrlBytes - 1024) / stage_bytes));
+    x->smem_bytes = kSmemCtrlBytes + 1024 + x->stages * stage_bytes;
+
+    const int B = cfg->B;
+    const size_t np = 2ull * B * x->slots_stride;
+    int rc = EAD_OK;
+    auto fail = [&](int code) {
+        ead_destroy(x);
+        return code;
+    };
+    if (x->stages < 2) return fail(EAD_ECUDA);
+    if (cudaStreamCreateWithFlags(&x->cap_stream, cudaStreamNonBlocking) != cudaSuccess) return fail(EAD_ECUDA);
+    if (cudaMalloc(&x->ctl, sizeof(StepCtl)) != cudaSuccess || cudaMalloc(&x->args, sizeof(RunArgs)) != cudaSuccess ||
+        cudaMalloc(&x->flag, B) != cudaSuccess || cudaMalloc(&x->c, 4ull * B) != cudaSuccess ||
+        cudaMalloc(&x->nfill, 4ull * B) != cudaSuccess || cudaMalloc(&x->perm, 8ull * B) != cudaSuccess ||
+        cudaMalloc(&x->ring, 4ull * B * cfg->w) != cudaSuccess ||
+        cudaMalloc(&x->hc[0], 2ull * B * cfg->H_small) != cudaSuccess ||
+        cudaMalloc(&x->hc[1], 2ull * B * cfg->H_large) != cudaSuccess ||
+        cudaMalloc(&x->part_m, 4 * np) != cudaSuccess || cudaMalloc(&x->part_s, 4 * np) != cudaSuccess ||
+        cudaMalloc(&x->part_t, 4 * np) != cudaSuccess || cudaMalloc(&x->part_i, 4 * np) != cudaSuccess)
+        return fail(EAD_ECUDA);
+    cudaMemsetAsync(x->ctl, 0, sizeof(StepCtl), x->stream);
+    cudaMemsetAsync(x->args, 0, sizeof(RunArgs), x->stream);
+    cudaMemsetAsync(x->perm, 0, 8ull * B, x->stream);
+    cudaMemsetAsync(x->hc[0], 0, 2ull * B * cfg->H_small, x->stream);
+    cudaMemsetAsync(x->hc[1], 0, 2ull * B * cfg->H_large, x->stream);
+    cudaMemsetAsync(x->part_m, 0, 4 * np, x->stream);
+    cudaMemsetAsync(x->part_s, 0, 4 * np, x->stream);
+    cudaMemsetAsync(x->part_t, 0, 4 * np, x->stream);
+    cudaMemsetAsync(x->part_i, 0, 4 * np, x->stream);
+
+    const uint32_t wbox = static_cast<uint32_t>(std::min(kTileN, (cfg->V + kUnit - 1) / kUnit * kUnit));
+    const int Hm[2] = {cfg->H_small, cfg->H_large};
+    for (int m = 0; m < 2; ++m) {
+        if (!encode_bf16_2d(&x->tmA[m], x->hc[m], B, Hm[m], x->a_rows) ||
+            !encode_bf16_2d(&x->tmW[m], x->W[m], cfg->V, Hm[m], wbox) ||
+            !encode_bf16_2d(&x->tmT[m], x->W[m], cfg->V, Hm[m], kUnit))
+            return fail(EAD_ECUDA);
+    }
+    if (cudaFuncSetAttribute(ead_lmhead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(x->smem_bytes)) != cudaSuccess)
+        return fail(EAD_ECUDA);
+    if (cudaFuncSetAttribute(ead_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * 4096) !=
+        cudaSuccess)
+        return fail(EAD_ECUDA);
+
+    rc = ead_reset(x);
+    if (rc != EAD_OK) return fail(rc);
+    rc = build_graph(x, 1, &x->g_one);
+    if (rc == EAD_OK) rc = build_graph(x, kGraphChunk, &x->g_chunk);
+    if (rc != EAD_OK) return fail(rc);
+    if (cudaStreamSynchronize(x->stream) != cudaSuccess) return fail(EAD_ECUDA);
+    *out = x;
+    return EAD_OK;
+}
+
+int ead_reset(ead_ctx *x)
+{
+    if (!x) return EAD_EINVALID_ARG;
+    const ead_config &c = x->cfg;
+    const int threads = 256;
+    ead_reset_kernel<<<(c.B + threads - 1) / threads, threads, 0, x->stream>>>(x->ctl, x->flag, x->c, x->nfill,
+                                                                              x->ring, c.B, c.w, c.start_model);
+    x->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? EAD_OK : EAD_ECUDA;
+}
+
+int ead_step(ead_ctx *x, const void *h_small, const void *h_large, int32_t *tok, float *H, float *Hbar,
+             uint8_t *model_used, uint8_t *next_model)
+{
+    if (!x || !h_small || !h_large) return EAD_EINVALID_ARG;
+    if (!aligned16(h_small) || !aligned16(h_large)) return EAD_EALIGNMENT;
+    int rc = set_args(x, h_small, h_large, tok, H, Hbar, model_used, next_model, x->stream);
+    if (rc != EAD_OK) return rc;
+    rc = enqueue_step(x, x->stream);
+    x->launches += 3;
+    return rc;
+}
+
+int ead_run(ead_ctx *x, int32_t T, const void *h_small_seq, const void *h_large_seq, int32_t *tok, float *H,
+            float *Hbar, uint8_t *model_used, uint8_t *next_model)
+{
+    if (!x || T < 0 || !h_small_seq || !h_large_seq) return EAD_EINVALID_ARG;
+    if (!aligned16(h_small_seq) || !aligned16(h_large_seq)) return EAD_EALIGNMENT;
+    if (T == 0) return EAD_OK;
+    return run_device(x, T, h_small_seq, h_large_seq, tok, H, Hbar, model_used, next_model);
+}
+
+int ead_run_host(ead_ctx *x, int32_t T, const void *h_small_seq, const void *h_large_seq, int32_t *tok, float *H,
+                 float *Hbar, uint8_t *model_used, uint8_t *next_model)
+{
+    if (!x || T < 0 || !h_small_seq || !h_large_seq) return EAD_EINVALID_ARG;
+    if (T == 0) return EAD_OK;
+    int rc = ensure_staging(x);
+    if (rc != EAD_OK) return rc;
+    const ead_config &c = x->cfg;
+    const int S = x->st_steps;
+    const OutLayout l = out_layout(S, c.B);
+    const size_t row_s = static_cast<size_t>(c.B) * c.H_small * 2, row_l = static_cast<size_t>(c.B) * c.H_large * 2;
+    const uint8_t *hs = static_cast<const uint8_t *>(h_small_seq), *hl = static_cast<const uint8_t *>(h_large_seq);
+    const int chunks = (T + S - 1) / S;
+    for (int k = 0; k < chunks; ++k) {
+        const int i = k & 1;
+        const int t0 = k * S, n = std::min(S, T - t0);
+        const size_t cells = static_cast<size_t>(n) * c.B;
+        // inputs of chunk k -> staging buffer i, once the compute that read it (chunk k-2) is done
+        if (k >= 2) EAD_CUDA(cudaStreamWaitEvent(x->in_stream, x->ev_comp[i], 0));
+        EAD_CUDA(cudaMemcpyAsync(x->st_h[i][0], hs + t0 * row_s, n * row_s, cudaMemcpyHostToDevice, x->in_stream));
+        EAD_CUDA(cudaMemcpyAsync(x->st_h[i][1], hl + t0 * row_l, n * row_l, cudaMemcpyHostToDevice, x->in_stream));
+        EAD_CUDA(cudaEventRecord(x->ev_in[i], x->in_stream));
+        // compute, once the inputs are in and the previous results of buffer i have been read back
+        EAD_CUDA(cudaStreamWaitEvent(x->stream, x->ev_in[i], 0));
+        if (k >= 2) EAD_CUDA(cudaStreamWaitEvent(x->stream, x->ev_out[i], 0));
+        uint8_t *o = static_cast<uint8_t *>(x->st_out[i]);
+        rc = run_device(x, n, x->st_h[i][0], x->st_h[i][1], reinterpret_cast<int32_t *>(o + l.off_tok),
+                        reinterpret_cast<float *>(o + l.off_H), reinterpret_cast<float *>(o + l.off_Hbar),
+                        o + l.off_used, o + l.off_next);
+        if (rc != EAD_OK) return rc;
+        EAD_CUDA(cudaEventRecord(x->ev_comp[i], x->stream));
+        // results of chunk k -> host
+        EAD_CUDA(cudaStreamWaitEvent(x->out_stream, x->ev_comp[i], 0));
+        const size_t o0 = static_cast<size_t>(t0) * c.B;
+        if (tok) EAD_CUDA(cudaMemcpyAsync(tok + o0, o + l.off_tok, 4 * cells, cudaMemcpyDeviceToHost, x->out_stream));
+        if (H) EAD_CUDA(cudaMemcpyAsync(H + o0, o + l.off_H, 4 * cells, cudaMemcpyDeviceToHost, x->out_stream));
+        if (Hbar) EAD_CUDA(cudaMemcpyAsync(Hbar + o0, o + l.off_Hbar, 4 * cells, cudaMemcpyDeviceToHost, x->out_stream));
+        if (model_used)
+            EAD_CUDA(cudaMemcpyAsync(model_used + o0, o + l.off_used, cells, cudaMemcpyDeviceToHost, x->out_stream));
+        if (next_model)
+            EAD_CUDA(cudaMemcpyAsync(next_model + o0, o + l.off_next, cells, cudaMemcpyDeviceToHost, x->out_stream));
+        EAD_CUDA(cudaEventRecord(x->ev_out[i], x->out_stream));
+    }
+    EAD_CUDA(cudaStreamSynchronize(x->out_stream));
+    EAD_CUDA(cudaStreamSynchronize(x->stream));
+    return EAD_OK;
+}
+
+int ead_status(ead_ctx *x, uint32_t *status_word)
+{
+    if (!x) return EAD_EINVALID_ARG;
+    EAD_CUDA(cudaStreamSynchronize(x->stream));
+    StepCtl h{};
+    EAD_CUDA(cudaMemcpy(&h, x->ctl, sizeof h, cudaMemcpyDeviceToHost));
+    if (status_word) *status_word = h.status;
+    return (h.status & (kStatusWaitExpired | kStatusBadCount)) ? EAD_EDEVICE_FAULT : EAD_OK;
+}
+
+size_t ead_state_size(const ead_ctx *x)
+{
+    if (!x) return 0;
+    const size_t B = x->cfg.B;
+    return sizeof(StateHeader) + B /*flag*/ + ((4 - B % 4) % 4) + 4 * B /*c*/ + 4 * B /*nfill*/ + 4 * B * x->cfg.w;
+}
+
+int ead_get_state(ead_ctx *x, void *blob, size_t size)
+{
+    if (!x || !blob) return EAD_EINVALID_ARG;
+    if (size != ead_state_size(x)) return EAD_ESTATE;
+    EAD_CUDA(cudaStreamSynchronize(x->stream));
+    const size_t B = x->cfg.B, pad = (4 - B % 4) % 4;
+    uint8_t *p = static_cast<uint8_t *>(blob);
+    StepCtl h{};
+    EAD_CUDA(cudaMemcpy(&h, x->ctl, sizeof h, cudaMemcpyDeviceToHost));
+    StateHeader hd{kStateMagic, x->cfg.B, x->cfg.w, h.step};
+    memcpy(p, &hd, sizeof hd);
+    p += sizeof hd;
+    EAD_CUDA(cudaMemcpy(p, x->flag, B, cudaMemcpyDeviceToHost));
+    memset(p + B, 0, pad);
+    p += B + pad;
+    EAD_CUDA(cudaMemcpy(p, x->c, 4 * B, cudaMemcpyDeviceToHost));
+    p += 4 * B;
+    EAD_CUDA(cudaMemcpy(p, x->nfill, 4 * B, cudaMemcpyDeviceToHost));
+    p += 4 * B;
+    EAD_CUDA(cudaMemcpy(p, x->ring, 4 * B * x->cfg.w, cudaMemcpyDeviceToHost));
+    return EAD_OK;
+}
+
+int ead_set_state(ead_ctx *x, const void *blob, size_t size)
+{
+    if (!x || !blob) return EAD_EINVALID_ARG;
+    if (size != ead_state_size(x)) return EAD_ESTATE;
+    const uint8_t *p = static_cast<const uint8_t *>(blob);
+    StateHeader hd;
+    memcpy(&hd, p, sizeof hd);
+    if (hd.magic != kStateMagic || hd.B != x->cfg.B || hd.w != x->cfg.w || hd.step < 0) return EAD_ESTATE;
+    EAD_CUDA(cudaStreamSynchronize(x->stream));
+    const size_t B = x->cfg.B, pad = (4 - B % 4) % 4;
+    p += sizeof hd;
+    for (size_t i = 0; i < B; ++i)
+        if (p[i] > 1) return EAD_ESTATE;
+    EAD_CUDA(cudaMemcpy(&x->ctl->step, &hd.step, 4, cudaMemcpyHostToDevice));
+    EAD_CUDA(cudaMemcpy(x->flag, p, B, cudaMemcpyHostToDevice));
+    p += B + pad;
+    EAD_CUDA(cudaMemcpy(x->c, p, 4 * B, cudaMemcpyHostToDevice));
+    p += 4 * B;
+    EAD_CUDA(cudaMemcpy(x->nfill, p, 4 * B, cudaMemcpyHostToDevice));
+    p += 4 * B;
+    EAD_CUDA(cudaMemcpy(x->ring, p, 4 * B * x->cfg.w, cudaMemcpyHostToDevice));
+    return EAD_OK;
+}
+
+int64_t ead_kernel_launches(const ead_ctx *x) { return x ? x->launches : 0; }
+
+int ead_launch_info(const ead_ctx *x, int32_t *info, int32_t n)
+{
+    if (!x || !info || n < 0) return EAD_EINVALID_ARG;
+    const int32_t v[4] = {x->G, x->stages, x->a_rows, static_cast<int32_t>(x->smem_bytes)};
+    for (int i = 0; i < n && i < 4; ++i) info[i] = v[i];
+    return EAD_OK;
+}
+
+void ead_destroy(ead_ctx *x)
+{
+    if (!x) return;
+    cudaSetDevice(x->cfg.device);
+    cudaStreamSynchronize(x->stream);
+    if (x->in_stream) cudaStreamSynchronize(x->in_stream);
+    if (x->out_stream) cudaStreamSynchronize(x->out_stream);
+    free_staging(x);
+    if (x->g_one) cudaGraphExecDestroy(x->g_one);
+    if (x->g_chunk) cudaGraphExecDestroy(x->g_chunk);
+    if (x->cap_stream) cudaStreamDestroy(x->cap_stream);
+    void *bufs[] = {x->ctl, x->args, x->flag, x->c, x->nfill, x->perm, x->ring, x->hc[0], x->hc[1],
+                    x->part_m, x->part_s, x->part_t, x->part_i};
+    for (void *b : bufs)
+        if (b) cudaFree(b);
+    cudaGetLastError();
+    delete x;
+}
+
+}  // extern "C"

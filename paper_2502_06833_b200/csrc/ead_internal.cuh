@@ -1,0 +1,93 @@
+// Device-side data shared by the kernels of the EAD gate step and the host API.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ead {
+
+constexpr int kTileN = 256;        // vocabulary columns per accumulator tile (MMA N)
+constexpr int kTileM = 128;        // batch rows per accumulator tile (MMA M = TMEM lanes)
+constexpr int kBlockK = 64;        // hidden elements per pipeline stage (128 B of bf16)
+constexpr int kUnit = 16;          // granularity of a CTA's vocabulary range (MMA N step)
+constexpr int kMaxStages = 8;
+constexpr int kWTileBytes = kTileN * kBlockK * 2;   // 32 KiB
+constexpr int kSmemCtrlBytes = 1024;
+constexpr int kLmheadThreads = 192;                 // TMA warp, MMA warp, 4 epilogue warps
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kNegSentinel = -1.0e30f;            // "no logit seen yet"; finite on purpose
+constexpr uint32_t kStatusNonFinite = 0x1u;
+constexpr uint32_t kStatusWaitExpired = 0x2u;
+constexpr uint32_t kStatusBadCount = 0x4u;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // bounded waits give up after 2 s
+
+// Step control block (device resident, one per context).
+struct StepCtl {
+    int32_t step;       // gate steps taken since the last reset
+    int32_t cur_t;      // copy of `step` taken by the compaction kernel for this step
+    int32_t n[2];       // rows served by the small / large head in this step
+    uint32_t status;    // sticky EAD_STATUS_* bits
+    int32_t pad[3];
+};
+
+// Caller buffers of the current ead_step / ead_run call (device resident so that a
+// captured graph does not freeze pointers).  Step `step - run_base` of the run reads
+// row block [idx * B, (idx + 1) * B) of the inputs and writes the same of the outputs.
+struct RunArgs {
+    const uint16_t *h[2];
+    int32_t *tok;
+    float *H;
+    float *Hbar;
+    uint8_t *used;
+    uint8_t *next;
+    int32_t run_base;
+    int32_t pad;
+};
+
+// How the CTAs of the LM-head kernel divide one head.  With n rows on the head there
+// are R = ceil(n / 128) row blocks; the first g * R CTAs (g = G / R) form R groups of
+// g CTAs; group member `slot` owns the vocabulary units [slot * U / g, (slot + 1) * U / g)
+// of 16 columns (U = ceil(V / 16)) for row block rb.  CTAs with the same slot work on
+// the same vocabulary range at about the same time, so a weight tile fetched by one is
+// an L2 hit for the others.
+struct HeadSplit {
+    int R, g, rb, slot, active;
+    int col_begin, col_end;    // multiples of 16; col_end may exceed V by < 16
+};
+
+__host__ __device__ inline HeadSplit split_head(int cta, int G, int n, int V)
+{
+    HeadSplit s;
+    s.R = (n + kTileM - 1) / kTileM;
+    if (n <= 0) {
+        s.g = 0; s.rb = 0; s.slot = 0; s.active = 0; s.col_begin = s.col_end = 0;
+        return s;
+    }
+    s.g = G / s.R;
+    if (s.g < 1) s.g = 1;      // only if R > G; then CTAs take several row blocks (not used: B <= 4096)
+    s.active = cta < s.g * s.R;
+    s.rb = cta % s.R;
+    s.slot = cta / s.R;
+    const long long U = (V + kUnit - 1) / kUnit;
+    s.col_begin = static_cast<int>((U * s.slot) / s.g) * kUnit;
+    s.col_end = static_cast<int>((U * (s.slot + 1)) / s.g) * kUnit;
+    if (!s.active) s.col_begin = s.col_end = 0;
+    return s;
+}
+
+struct LmheadParams {
+    int32_t V;
+    int32_t H[2];
+    int32_t a_rows;        // rows of the hidden-state TMA box (multiple of 8, <= 128)
+    int32_t stages;
+    int32_t slots_stride;  // partial slots per row (>= CTAs)
+    int32_t B;
+    const StepCtl *ctl;
+    StepCtl *ctl_rw;
+    float *part_m;         // [2][B][slots_stride] running max (nats)
+    float *part_s;         // sum of exp(z - m)
+    float *part_t;         // sum of exp(z - m) * (z - m) * log2(e)
+    int32_t *part_i;       // column of the max
+};
+
+}  // namespace ead

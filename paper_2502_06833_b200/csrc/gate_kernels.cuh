@@ -1,0 +1,217 @@
+// The integer / per-row kernels around the LM-head contraction:
+//   ead_compact_kernel     splits the batch by active model and gathers the active
+//                          model's hidden row of every sequence into a dense operand
+//   ead_merge_gate_kernel  merges the per-CTA partial statistics into the entropy of
+//                          Eq. 2 and the greedy token, then runs the window / dwell /
+//                          threshold part of Algorithm 1 (Eq. 3-4) and updates the state
+//   ead_set_args_kernel, ead_reset_kernel   bookkeeping
+#pragma once
+#include "ead_internal.cuh"
+
+namespace ead {
+
+constexpr int kCompactThreads = 256;
+constexpr int kGateThreads = 256;
+
+__global__ void ead_set_args_kernel(RunArgs *dst, RunArgs a, const StepCtl *ctl)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        a.run_base = ctl->step;
+        *dst = a;
+    }
+}
+
+__global__ void ead_reset_kernel(StepCtl *ctl, uint8_t *flag, int32_t *c, int32_t *nfill, float *ring,
+                                 int B, int w, int start_model)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i == 0) {
+        ctl->step = 0;
+        ctl->cur_t = 0;
+        ctl->n[0] = ctl->n[1] = 0;
+        ctl->status = 0;
+    }
+    if (i < B) {
+        flag[i] = static_cast<uint8_t>(start_model);
+        c[i] = 0;
+        nfill[i] = 0;
+    }
+    for (int k = i; k < B * w; k += gridDim.x * blockDim.x) ring[k] = 0.f;
+}
+
+// Stable partition of the rows by model flag.  Every CTA recomputes the (tiny) scan
+// over the B flags and then copies the rows b = blockIdx.x, blockIdx.x + gridDim.x, ...
+// perm[m * B + r] = original row of compacted row r of head m.
+__global__ void __launch_bounds__(kCompactThreads)
+ead_compact_kernel(StepCtl *ctl, const RunArgs *args, const uint8_t *flag, int B, int Hs, int Hl,
+                   uint16_t *hc_s, uint16_t *hc_l, int32_t *perm)
+{
+    extern __shared__ int32_t pos_sh[];          // [B]: position | model << 30
+    __shared__ int32_t warp_tot[kCompactThreads / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int step = ctl->step;
+    const int idx = step - args->run_base;
+
+    const int per = (B + kCompactThreads - 1) / kCompactThreads;
+    const int b0 = min(B, tid * per), b1 = min(B, b0 + per);
+    int cnt = 0;
+    for (int b = b0; b < b1; ++b) cnt += flag[b] ? 1 : 0;
+    int incl = cnt;                               // inclusive scan of the large-model counts
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    int before = 0, total_large = 0;
+#pragma unroll
+    for (int k = 0; k < kCompactThreads / 32; ++k) {
+        const int v = warp_tot[k];
+        if (k < warp) before += v;
+        total_large += v;
+    }
+    int pos_l = before + incl - cnt;              // large rows before b0
+    int pos_s = b0 - pos_l;                       // small rows before b0
+    for (int b = b0; b < b1; ++b) {
+        const int f = flag[b] ? 1 : 0;
+        const int pos = f ? pos_l++ : pos_s++;
+        pos_sh[b] = pos | (f << 30);
+        if (blockIdx.x == 0) perm[f * B + pos] = b;
+    }
+    if (blockIdx.x == 0 && tid == 0) {
+        ctl->n[0] = B - total_large;
+        ctl->n[1] = total_large;
+        ctl->cur_t = step;
+    }
+    __syncthreads();
+
+    for (int b = blockIdx.x; b < B; b += gridDim.x) {
+        const int e = pos_sh[b];
+        const int f = e >> 30, pos = e & 0x3fffffff;
+        const int H = f ? Hl : Hs;
+        const uint4 *src = reinterpret_cast<const uint4 *>(args->h[f] + (static_cast<size_t>(idx) * B + b) * H);
+        uint4 *dst = reinterpret_cast<uint4 *>((f ? hc_l : hc_s) + static_cast<size_t>(pos) * H);
+        for (int k = tid; k < H / 8; k += kCompactThreads) dst[k] = __ldg(src + k);
+    }
+}
+
+struct Partial {
+    float m, s, t;
+    int idx;
+};
+
+// Combines the statistics of two disjoint column sets (see lmhead_kernel.cuh for the
+// meaning of m, s, t).  Equal maxima keep the lower column.
+__device__ __forceinline__ Partial merge_partial(const Partial &a, const Partial &b)
+{
+    Partial r;
+    r.m = fmaxf(a.m, b.m);
+    const float da = (a.m - r.m) * kLog2e, db = (b.m - r.m) * kLog2e;
+    const float ea = exp2f(da), eb = exp2f(db);
+    r.s = ea * a.s + eb * b.s;
+    r.t = ea * fmaf(da, a.s, a.t) + eb * fmaf(db, b.s, b.t);
+    if (a.m > b.m) r.idx = a.idx;
+    else if (b.m > a.m) r.idx = b.idx;
+    else r.idx = min(a.idx, b.idx);
+    return r;
+}
+
+struct GateParams {
+    int32_t B, V, w, d_min, unit, G, slots_stride;
+    float tau;
+    StepCtl *ctl;
+    const RunArgs *args;
+    const float *part_m, *part_s, *part_t;
+    const int32_t *part_i;
+    const int32_t *perm;
+    uint8_t *flag;
+    int32_t *c;
+    int32_t *nfill;
+    float *ring;
+};
+
+// One warp per compacted row.
+__global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const GateParams p)
+{
+    const int lane = threadIdx.x & 31;
+    const int i = blockIdx.x * (kGateThreads / 32) + (threadIdx.x >> 5);
+    const int n0 = p.ctl->n[0], n1 = p.ctl->n[1];
+    const int t_step = p.ctl->cur_t;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        if (n0 + n1 != p.B) atomicOr(&p.ctl->status, kStatusBadCount);
+        p.ctl->step = t_step + 1;                 // nobody in this kernel reads `step`
+    }
+    if (i >= p.B || n0 + n1 != p.B) return;
+    const int m = i < n0 ? 0 : 1;
+    const int r = m ? i - n0 : i;
+    const int n_m = m ? n1 : n0;
+    const int R = (n_m + kTileM - 1) / kTileM;
+    int g = p.G / R;
+    if (g < 1) g = 1;
+
+    // ---- cross-CTA merge, fixed order: each lane folds its slots in ascending
+    //      order, then a butterfly over the lanes (no float atomics: deterministic)
+    const size_t base = (static_cast<size_t>(m) * p.B + r) * p.slots_stride;
+    Partial acc{kNegSentinel, 0.f, 0.f, 0x7fffffff};
+    for (int s = lane; s < g; s += 32) {
+        const Partial q{p.part_m[base + s], p.part_s[base + s], p.part_t[base + s], p.part_i[base + s]};
+        acc = merge_partial(acc, q);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Partial q;
+        q.m = __shfl_xor_sync(0xffffffffu, acc.m, o);
+        q.s = __shfl_xor_sync(0xffffffffu, acc.s, o);
+        q.t = __shfl_xor_sync(0xffffffffu, acc.t, o);
+        q.idx = __shfl_xor_sync(0xffffffffu, acc.idx, o);
+        acc = merge_partial(acc, q);
+    }
+    if (lane != 0) return;
+
+    // ---- Eq. 2 in the fused form  H = ln Z - E_p[z] = ln s - t / (s log2 e)   (nats)
+    float H = logf(acc.s) - acc.t / (acc.s * kLog2e);
+    const bool finite = isfinite(H) && acc.s > 0.f;
+    if (H < 0.f) H = 0.f;                         // rounding can leave -1e-7 for a one-hot row
+    if (p.unit == 1) H *= kLog2e;                 // bits, as Eq. 2 is printed
+
+    const int b = p.perm[m * p.B + r];
+    const size_t o = static_cast<size_t>(t_step - p.args->run_base) * p.B + b;
+    int model = p.flag[b];
+    if (!finite) {
+        // non-finite logits: report, leave window, counter and model untouched
+        atomicOr(&p.ctl->status, kStatusNonFinite);
+        if (p.args->tok) p.args->tok[o] = -1;
+        if (p.args->H) p.args->H[o] = __int_as_float(0x7fc00000);
+        if (p.args->Hbar) p.args->Hbar[o] = __int_as_float(0x7fc00000);
+        if (p.args->used) p.args->used[o] = static_cast<uint8_t>(model);
+        if (p.args->next) p.args->next[o] = static_cast<uint8_t>(model);
+        return;
+    }
+    // ---- Algorithm 1: append H_t to W; mean of the last w entries (those present)
+    int nf = p.nfill[b];
+    float *ring = p.ring + static_cast<size_t>(b) * p.w;
+    ring[nf % p.w] = H;
+    nf += 1;
+    const int cnt = nf < p.w ? nf : p.w;
+    float sum = 0.f;
+    for (int k = 0; k < cnt; ++k) sum += ring[k];
+    const float Hbar = sum / static_cast<float>(cnt);
+    // ---- c <- c + 1; Eq. 4
+    int c = p.c[b] + 1;
+    const int used = model;
+    if (c >= p.d_min) {
+        if (model == 0 && Hbar > p.tau) { model = 1; c = 0; }
+        else if (model == 1 && Hbar <= p.tau) { model = 0; c = 0; }
+    }
+    p.nfill[b] = nf;
+    p.c[b] = c;
+    p.flag[b] = static_cast<uint8_t>(model);
+    if (p.args->tok) p.args->tok[o] = acc.idx;
+    if (p.args->H) p.args->H[o] = H;
+    if (p.args->Hbar) p.args->Hbar[o] = Hbar;
+    if (p.args->used) p.args->used[o] = static_cast<uint8_t>(used);
+    if (p.args->next) p.args->next[o] = static_cast<uint8_t>(model);
+}
+
+}  // namespace ead
