@@ -317,6 +317,9 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     x->smem_bytes = kSmemCtrlBytes + 1024 + x->stages * stage_bytes;
 
     const int B = cfg->B;
+    // compacted operands are padded to whole row blocks (zeros) so that no TMA box of
+    // hidden rows reaches past the tensor
+    const size_t Bpad = (static_cast<size_t>(B) + kTileM - 1) / kTileM * kTileM;
     const size_t np = 2ull * B * x->slots_stride;
     int rc = EAD_OK;
     auto fail = [&](int code) {
@@ -329,16 +332,16 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
         cudaMalloc(&x->flag, B) != cudaSuccess || cudaMalloc(&x->c, 4ull * B) != cudaSuccess ||
         cudaMalloc(&x->nfill, 4ull * B) != cudaSuccess || cudaMalloc(&x->perm, 8ull * B) != cudaSuccess ||
         cudaMalloc(&x->ring, 4ull * B * cfg->w) != cudaSuccess ||
-        cudaMalloc(&x->hc[0], 2ull * B * cfg->H_small) != cudaSuccess ||
-        cudaMalloc(&x->hc[1], 2ull * B * cfg->H_large) != cudaSuccess ||
+        cudaMalloc(&x->hc[0], 2ull * Bpad * cfg->H_small) != cudaSuccess ||
+        cudaMalloc(&x->hc[1], 2ull * Bpad * cfg->H_large) != cudaSuccess ||
         cudaMalloc(&x->part_m, 4 * np) != cudaSuccess || cudaMalloc(&x->part_s, 4 * np) != cudaSuccess ||
         cudaMalloc(&x->part_t, 4 * np) != cudaSuccess || cudaMalloc(&x->part_i, 4 * np) != cudaSuccess)
         return fail(EAD_ECUDA);
     cudaMemsetAsync(x->ctl, 0, sizeof(StepCtl), x->stream);
     cudaMemsetAsync(x->args, 0, sizeof(RunArgs), x->stream);
     cudaMemsetAsync(x->perm, 0, 8ull * B, x->stream);
-    cudaMemsetAsync(x->hc[0], 0, 2ull * B * cfg->H_small, x->stream);
-    cudaMemsetAsync(x->hc[1], 0, 2ull * B * cfg->H_large, x->stream);
+    cudaMemsetAsync(x->hc[0], 0, 2ull * Bpad * cfg->H_small, x->stream);
+    cudaMemsetAsync(x->hc[1], 0, 2ull * Bpad * cfg->H_large, x->stream);
     cudaMemsetAsync(x->part_m, 0, 4 * np, x->stream);
     cudaMemsetAsync(x->part_s, 0, 4 * np, x->stream);
     cudaMemsetAsync(x->part_t, 0, 4 * np, x->stream);
@@ -347,7 +350,7 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     const uint32_t wbox = static_cast<uint32_t>(std::min(kTileN, (cfg->V + kUnit - 1) / kUnit * kUnit));
     const int Hm[2] = {cfg->H_small, cfg->H_large};
     for (int m = 0; m < 2; ++m) {
-        if (!encode_bf16_2d(&x->tmA[m], x->hc[m], B, Hm[m], x->a_rows) ||
+        if (!encode_bf16_2d(&x->tmA[m], x->hc[m], Bpad, Hm[m], x->a_rows) ||
             !encode_bf16_2d(&x->tmW[m], x->W[m], cfg->V, Hm[m], wbox) ||
             !encode_bf16_2d(&x->tmT[m], x->W[m], cfg->V, Hm[m], kUnit))
             return fail(EAD_ECUDA);
