@@ -122,6 +122,18 @@ int ead_run(ead_ctx *ctx, int32_t T, const void *h_small_seq, const void *h_larg
 int ead_run_host(ead_ctx *ctx, int32_t T, const void *h_small_seq, const void *h_large_seq,
                  int32_t *tok, float *H, float *Hbar, uint8_t *model_used, uint8_t *next_model);
 
+/*
+ * The same T steps as ead_run, launched kernel by kernel (no graph replay) with
+ * CUDA events around every kernel on cfg.stream, to attribute device time.
+ *   kernel_ms  host, float [3]: summed device time in milliseconds of the
+ *              compaction, LM-head and merge+gate kernels over the T steps
+ * Synchronous (waits for the stream).  Results are identical to ead_run; the
+ * event records make it slower, so it is a measurement aid, not the fast path.
+ */
+int ead_run_timed(ead_ctx *ctx, int32_t T, const void *h_small_seq, const void *h_large_seq,
+                  int32_t *tok, float *H, float *Hbar, uint8_t *model_used, uint8_t *next_model,
+                  float *kernel_ms);
+
 /* Back to Algorithm 1's initial state (empty window, c = 0, start model) and a
  * cleared status word.  Asynchronous. */
 int ead_reset(ead_ctx *ctx);

@@ -23,7 +23,7 @@ EAD_STATUS_NONFINITE = 0x1
 EAD_STATUS_WAIT_EXPIRED = 0x2
 EAD_STATUS_BAD_COUNT = 0x4
 
-SYMBOLS = ["ead_create", "ead_step", "ead_run", "ead_run_host", "ead_reset", "ead_status",
+SYMBOLS = ["ead_create", "ead_step", "ead_run", "ead_run_host", "ead_run_timed", "ead_reset", "ead_status",
            "ead_state_size", "ead_get_state", "ead_set_state", "ead_kernel_launches",
            "ead_launch_info", "ead_destroy", "ead_strerror"]
 
@@ -60,6 +60,9 @@ def lib() -> C.CDLL:
             f = getattr(L, name)
             f.restype = C.c_int
             f.argtypes = [vp, C.c_int32, vp, vp, i32p, f32p, f32p, u8p, u8p]
+        L.ead_run_timed.restype = C.c_int
+        L.ead_run_timed.argtypes = [vp, C.c_int32, vp, vp, i32p, f32p, f32p, u8p, u8p,
+                                    C.POINTER(C.c_float)]
         L.ead_reset.restype = C.c_int
         L.ead_reset.argtypes = [vp]
         L.ead_status.restype = C.c_int
@@ -129,6 +132,15 @@ def ead_run_host(ctx, T, h_small_seq, h_large_seq, tok=None, H=None, Hbar=None, 
     """All buffers are HOST memory (numpy arrays or CPU tensors, ideally pinned)."""
     _check(lib().ead_run_host(ctx, int(T), _ptr(h_small_seq), _ptr(h_large_seq), _ptr(tok), _ptr(H),
                               _ptr(Hbar), _ptr(model_used), _ptr(next_model)), "ead_run_host")
+
+
+def ead_run_timed(ctx, T, h_small_seq, h_large_seq, tok=None, H=None, Hbar=None, model_used=None,
+                  next_model=None) -> dict:
+    """ead_run with CUDA events around every kernel; returns summed milliseconds per kernel."""
+    ms = (C.c_float * 3)()
+    _check(lib().ead_run_timed(ctx, int(T), _ptr(h_small_seq), _ptr(h_large_seq), _ptr(tok), _ptr(H),
+                               _ptr(Hbar), _ptr(model_used), _ptr(next_model), ms), "ead_run_timed")
+    return dict(compact_ms=ms[0], lmhead_ms=ms[1], merge_gate_ms=ms[2])
 
 
 def ead_reset(ctx):

@@ -100,13 +100,16 @@ namespace {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// The three kernels of one gate step, in stream order.
-int enqueue_step(ead_ctx *x, cudaStream_t s)
+// The three kernels of one gate step, in stream order.  With `ev` (4 events) the
+// boundaries between the kernels are recorded for timing.
+int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
 {
     const ead_config &c = x->cfg;
     const int cgrid = std::min(c.B, 4 * x->G);
+    if (ev) cudaEventRecord(ev[0], s);
     ead_compact_kernel<<<cgrid, kCompactThreads, static_cast<size_t>(c.B) * sizeof(int32_t), s>>>(
         x->ctl, x->args, x->flag, c.B, c.H_small, c.H_large, x->hc[0], x->hc[1], x->perm);
+    if (ev) cudaEventRecord(ev[1], s);
 
     LmheadParams lp{};
     lp.V = c.V;
@@ -124,6 +127,7 @@ int enqueue_step(ead_ctx *x, cudaStream_t s)
     lp.part_i = x->part_i;
     ead_lmhead_kernel<<<x->G, kLmheadThreads, x->smem_bytes, s>>>(x->tmA[0], x->tmA[1], x->tmW[0], x->tmW[1],
                                                                   x->tmT[0], x->tmT[1], lp);
+    if (ev) cudaEventRecord(ev[2], s);
 
     GateParams gp{};
     gp.B = c.B;
@@ -147,6 +151,7 @@ int enqueue_step(ead_ctx *x, cudaStream_t s)
     gp.ring = x->ring;
     const int rows_per_block = kGateThreads / 32;
     ead_merge_gate_kernel<<<(c.B + rows_per_block - 1) / rows_per_block, kGateThreads, 0, s>>>(gp);
+    if (ev) cudaEventRecord(ev[3], s);
     return cudaGetLastError() == cudaSuccess ? EAD_OK : EAD_ECUDA;
 }
 
@@ -402,6 +407,39 @@ int ead_run(ead_ctx *x, int32_t T, const void *h_small_seq, const void *h_large_
     if (!aligned16(h_small_seq) || !aligned16(h_large_seq)) return EAD_EALIGNMENT;
     if (T == 0) return EAD_OK;
     return run_device(x, T, h_small_seq, h_large_seq, tok, H, Hbar, model_used, next_model);
+}
+
+int ead_run_timed(ead_ctx *x, int32_t T, const void *h_small_seq, const void *h_large_seq, int32_t *tok, float *H,
+                  float *Hbar, uint8_t *model_used, uint8_t *next_model, float *kernel_ms)
+{
+    if (!x || T < 0 || !h_small_seq || !h_large_seq || !kernel_ms) return EAD_EINVALID_ARG;
+    if (!aligned16(h_small_seq) || !aligned16(h_large_seq)) return EAD_EALIGNMENT;
+    kernel_ms[0] = kernel_ms[1] = kernel_ms[2] = 0.f;
+    if (T == 0) return EAD_OK;
+    constexpr int kBatch = 64;                 // steps between synchronisations
+    std::vector<cudaEvent_t> ev(4 * kBatch, nullptr);
+    int rc = EAD_OK;
+    for (auto &e : ev)
+        if (cudaEventCreate(&e) != cudaSuccess) rc = EAD_ECUDA;
+    if (rc == EAD_OK) rc = set_args(x, h_small_seq, h_large_seq, tok, H, Hbar, model_used, next_model, x->stream);
+    double acc[3] = {0, 0, 0};
+    for (int t0 = 0; t0 < T && rc == EAD_OK; t0 += kBatch) {
+        const int n = std::min(kBatch, T - t0);
+        for (int i = 0; i < n && rc == EAD_OK; ++i) rc = enqueue_step(x, x->stream, &ev[4 * i]);
+        x->launches += 3ll * n;
+        if (rc == EAD_OK && cudaStreamSynchronize(x->stream) != cudaSuccess) rc = EAD_ECUDA;
+        for (int i = 0; i < n && rc == EAD_OK; ++i)
+            for (int k = 0; k < 3; ++k) {
+                float ms = 0.f;
+                if (cudaEventElapsedTime(&ms, ev[4 * i + k], ev[4 * i + k + 1]) != cudaSuccess) rc = EAD_ECUDA;
+                acc[k] += ms;
+            }
+    }
+    for (auto &e : ev)
+        if (e) cudaEventDestroy(e);
+    for (int k = 0; k < 3; ++k) kernel_ms[k] = static_cast<float>(acc[k]);
+    if (rc != EAD_OK) cudaGetLastError();
+    return rc;
 }
 
 int ead_run_host(ead_ctx *x, int32_t T, const void *h_small_seq, const void *h_large_seq, int32_t *tok, float *H,
