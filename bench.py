@@ -157,7 +157,7 @@ def oracle_sample(cfg, wl, budget_s: float, max_steps: int, skip: int):
     skip = min(skip, wl.T - 1)
     t_skip, _ = timed(skip)
     t_probe, _ = timed(skip + 1)
-    per_step = max(t_probe - t_skip, 1e-4)
+    per_step = max(t_probe - t_skip, t_skip / max(skip, 1), 1e-4)
     n = int(max(1, min(max_steps, wl.T - skip, (budget_s - t_skip) / per_step)))
     t_all, out = timed(skip + n)
     dt = max(t_all - t_skip, 1e-9)
