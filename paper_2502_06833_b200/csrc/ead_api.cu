@@ -360,8 +360,10 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
             !encode_bf16_2d(&x->tmT[m], x->W[m], cfg->V, Hm[m], kUnit))
             return fail(EAD_ECUDA);
     }
+    // the attribute belongs to the kernel on this device, not to the context: ask for the
+    // device maximum so that contexts with different stage counts can coexist
     if (cudaFuncSetAttribute(ead_lmhead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(x->smem_bytes)) != cudaSuccess)
+                             static_cast<int>(smem_max)) != cudaSuccess)
         return fail(EAD_ECUDA);
     if (cudaFuncSetAttribute(ead_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * 4096) !=
         cudaSuccess)
