@@ -46,6 +46,7 @@ extern "C" {
 #define EAD_EUNSUPPORTED_ARCH (-4)  /* device is not sm_100                                 */
 #define EAD_EDEVICE_FAULT     (-5)  /* the device status word reports a kernel-side error   */
 #define EAD_ESTATE            (-6)  /* state blob of the wrong size or version              */
+#define EAD_ELIMIT            (-7)  /* size beyond a fixed built-in limit (see EAD_STATIC_*)  */
 
 /* Bits of the device status word (ead_status). */
 #define EAD_STATUS_NONFINITE   0x1u /* some row saw a NaN / infinite logit (row gets H = NaN) */
@@ -165,6 +166,48 @@ int ead_launch_info(const ead_ctx *ctx, int32_t *info, int32_t n);
 
 /* Waits for outstanding work and frees everything the context owns.  NULL is allowed. */
 void ead_destroy(ead_ctx *ctx);
+
+/*
+ * Entropy and greedy token of one LM head for a dense batch, WITHOUT any allocation.
+ * (The paper has no counterpart: this is a service entry point of the library; what it
+ * computes per row is Eq. 1-2 and the arg max, exactly as one ead_step does for rows
+ * that are on that head.)
+ *
+ * For callers that are not allowed to allocate device memory: code that runs while the
+ * framework's allocator is frozen (inside a memory-planned inference engine, under a
+ * fixed memory budget that has already been handed out, or in a latency-critical section
+ * where cudaMalloc's implicit device synchronisation is unacceptable).  ead_create and
+ * ead_run_host call cudaMalloc; this function calls neither cudaMalloc nor cudaFree nor
+ * any allocating library routine.  Its scratch memory (per-CTA partial statistics, a
+ * padded copy of the hidden rows, a control block) lives in one array compiled into the
+ * library, about 2.4 MB, which every GPU that loads the library holds until the process
+ * exits.  That fixes the limits:
+ *     B <= EAD_STATIC_MAX_B (128),  H <= EAD_STATIC_MAX_H (8192),  H a multiple of 8.
+ * Larger sizes are rejected with EAD_ELIMIT before anything is launched.
+ *
+ *   W        dev, bf16 [V, H] row major, 16-byte aligned (borrowed, read only)
+ *   h        dev, bf16 [B, H] row major, 16-byte aligned: one hidden row per sequence
+ *   tok      dev, int32 [B]: greedy token, lowest index among equal maxima (-1 for a row
+ *            with non-finite logits); may be NULL
+ *   H_out    dev, float [B]: entropy in nats (NaN for a row with non-finite logits); may be NULL
+ *   status   dev, uint32 [1]: receives EAD_STATUS_* bits of this call; may be NULL
+ *   device   CUDA device ordinal; made current by the call
+ *   stream   cudaStream_t to enqueue on; NULL = legacy default stream
+ *
+ * Asynchronous: three kernels are enqueued on `stream`.  The first call on a device also
+ * looks up the device address of the built-in array and the device's limits; make that
+ * first call outside any stream capture.
+ * Every call on a device uses the SAME array.  The call rewrites all of it that it later
+ * reads (nothing of an earlier call leaks into the result), but two calls whose kernels
+ * overlap on the GPU (different streams, no dependency) race on it: keep calls on one
+ * device ordered.  Not thread safe with respect to other calls on the same device.
+ * Errors: EAD_EINVALID_ARG, EAD_EALIGNMENT, EAD_ELIMIT, EAD_EUNSUPPORTED_ARCH, EAD_ECUDA.
+ */
+#define EAD_STATIC_MAX_B 128
+#define EAD_STATIC_MAX_H 8192
+int ead_head_entropy_static(const void *W, const void *h, int32_t B, int32_t V, int32_t H,
+                            int32_t *tok, float *H_out, uint32_t *status, int32_t device,
+                            void *stream);
 
 /* Static, NUL-terminated description of an EAD_E* code. */
 const char *ead_strerror(int code);

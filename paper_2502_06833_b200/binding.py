@@ -19,13 +19,16 @@ EAD_ECUDA = -3
 EAD_EUNSUPPORTED_ARCH = -4
 EAD_EDEVICE_FAULT = -5
 EAD_ESTATE = -6
+EAD_ELIMIT = -7
+EAD_STATIC_MAX_B = 128
+EAD_STATIC_MAX_H = 8192
 EAD_STATUS_NONFINITE = 0x1
 EAD_STATUS_WAIT_EXPIRED = 0x2
 EAD_STATUS_BAD_COUNT = 0x4
 
 SYMBOLS = ["ead_create", "ead_step", "ead_run", "ead_run_host", "ead_run_timed", "ead_reset", "ead_status",
            "ead_state_size", "ead_get_state", "ead_set_state", "ead_kernel_launches",
-           "ead_launch_info", "ead_destroy", "ead_strerror"]
+           "ead_launch_info", "ead_destroy", "ead_strerror", "ead_head_entropy_static"]
 
 
 class EadConfig(C.Structure):
@@ -79,6 +82,9 @@ def lib() -> C.CDLL:
         L.ead_launch_info.argtypes = [vp, C.POINTER(C.c_int32), C.c_int32]
         L.ead_destroy.restype = None
         L.ead_destroy.argtypes = [vp]
+        L.ead_head_entropy_static.restype = C.c_int
+        L.ead_head_entropy_static.argtypes = [vp, vp, C.c_int32, C.c_int32, C.c_int32, i32p, f32p, vp,
+                                              C.c_int32, vp]
         L.ead_strerror.restype = C.c_char_p
         L.ead_strerror.argtypes = [C.c_int]
         _lib = L
@@ -179,6 +185,16 @@ def ead_launch_info(ctx) -> dict:
     a = (C.c_int32 * 4)()
     _check(lib().ead_launch_info(ctx, a, 4), "ead_launch_info")
     return dict(ctas=a[0], stages=a[1], a_rows=a[2], smem_bytes=a[3])
+
+
+def ead_head_entropy_static(W, h, B, V, H, tok=None, H_out=None, status=None, device=0, stream=0):
+    """Entropy (nats) and greedy token of one LM head for a dense batch, for callers that
+    may not allocate device memory: the library uses a scratch array compiled into it
+    (B <= EAD_STATIC_MAX_B, H <= EAD_STATIC_MAX_H).  All buffers are device memory owned
+    by the caller; asynchronous on ``stream``."""
+    _check(lib().ead_head_entropy_static(_ptr(W), _ptr(h), int(B), int(V), int(H), _ptr(tok),
+                                         _ptr(H_out), _ptr(status), int(device),
+                                         C.c_void_p(int(stream))), "ead_head_entropy_static")
 
 
 def ead_destroy(ctx) -> None:

@@ -8,6 +8,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -286,6 +287,7 @@ const char *ead_strerror(int code)
         case EAD_EUNSUPPORTED_ARCH: return "device is not sm_100";
         case EAD_EDEVICE_FAULT: return "device status word reports a kernel-side error";
         case EAD_ESTATE: return "state blob does not match this context";
+        case EAD_ELIMIT: return "size exceeds a built-in limit (EAD_STATIC_MAX_B / EAD_STATIC_MAX_H)";
         default: return "unknown error";
     }
 }
@@ -586,3 +588,175 @@ void ead_destroy(ead_ctx *x)
 }
 
 }  // extern "C"
+
+// =====================================================================================
+// Allocation-free entry point.  Everything below is independent of ead_ctx: its scratch
+// is the file-scope device array g_static_scratch, shared by all calls on a device.
+// =====================================================================================
+namespace {
+
+constexpr int kStaticSlots = 160;          // partial slots per row (>= CTAs launched)
+constexpr int kStaticMaxDevices = 64;
+
+// Layout of the built-in scratch array.
+struct StaticScratch {
+    StepCtl ctl;
+    unsigned char pad[256 - sizeof(StepCtl)];
+    float part_m[EAD_STATIC_MAX_B * kStaticSlots];
+    float part_s[EAD_STATIC_MAX_B * kStaticSlots];
+    float part_t[EAD_STATIC_MAX_B * kStaticSlots];
+    int32_t part_i[EAD_STATIC_MAX_B * kStaticSlots];
+    uint16_t hidden[EAD_STATIC_MAX_B * EAD_STATIC_MAX_H];   // padded copy of the hidden rows
+};
+
+// In host code this name is only a handle for cudaGetSymbolAddress, not a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
+
+struct StaticDevice {
+    bool ready = false;
+    StaticScratch *scratch = nullptr;      // device address of g_static_scratch on this device
+    int sms = 0;
+    int smem_optin = 0;
+};
+StaticDevice g_static_dev[kStaticMaxDevices];
+std::mutex g_static_mu;
+
+// Copies the caller's rows into the padded operand (rows B .. a_rows-1 are cleared, so the
+// TMA box never reads what an earlier call left there) and writes the control block.
+__global__ void ead_static_stage_kernel(StaticScratch *sc, const uint16_t *h, int B, int H, int a_rows)
+{
+    const int row = blockIdx.x;
+    if (row == 0 && threadIdx.x == 0) {
+        sc->ctl.step = 0;
+        sc->ctl.cur_t = 0;
+        sc->ctl.n[0] = B;
+        sc->ctl.n[1] = 0;
+        sc->ctl.status = 0;
+    }
+    if (row >= a_rows) return;
+    uint4 *dst = reinterpret_cast<uint4 *>(sc->hidden + static_cast<size_t>(row) * H);
+    if (row < B) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(h + static_cast<size_t>(row) * H);
+        for (int k = threadIdx.x; k < H / 8; k += blockDim.x) dst[k] = __ldg(src + k);
+    } else {
+        for (int k = threadIdx.x; k < H / 8; k += blockDim.x) dst[k] = make_uint4(0, 0, 0, 0);
+    }
+}
+
+// One warp per row: merge the G per-CTA partials in fixed order, then Eq. 2 in the fused
+// form and the arg max.
+__global__ void __launch_bounds__(kGateThreads)
+ead_static_merge_kernel(const StaticScratch *sc, int B, int G, int32_t *tok, float *H_out, uint32_t *status)
+{
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.x * (kGateThreads / 32) + (threadIdx.x >> 5);
+    if (r >= B) return;
+    const size_t base = static_cast<size_t>(r) * kStaticSlots;
+    Partial acc{kNegSentinel, 0.f, 0.f, 0x7fffffff};
+    for (int s = lane; s < G; s += 32) {
+        const Partial q{sc->part_m[base + s], sc->part_s[base + s], sc->part_t[base + s], sc->part_i[base + s]};
+        acc = merge_partial(acc, q);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Partial q;
+        q.m = __shfl_xor_sync(0xffffffffu, acc.m, o);
+        q.s = __shfl_xor_sync(0xffffffffu, acc.s, o);
+        q.t = __shfl_xor_sync(0xffffffffu, acc.t, o);
+        q.idx = __shfl_xor_sync(0xffffffffu, acc.idx, o);
+        acc = merge_partial(acc, q);
+    }
+    if (lane != 0) return;
+    float H = logf(acc.s) - acc.t / (acc.s * kLog2e);
+    const bool finite = isfinite(H) && acc.s > 0.f;
+    if (H < 0.f) H = 0.f;
+    uint32_t st = sc->ctl.status;
+    if (!finite) st |= kStatusNonFinite;
+    if (tok) tok[r] = finite ? acc.idx : -1;
+    if (H_out) H_out[r] = finite ? H : __int_as_float(0x7fc00000);
+    if (status && st) atomicOr(status, st);
+}
+
+__global__ void ead_static_clear_status_kernel(uint32_t *status)
+{
+    if (status) *status = 0;
+}
+
+// Once per device, with that device current: device address of the array, device limits.
+int static_device_setup(int device, StaticDevice **out)
+{
+    if (device < 0 || device >= kStaticMaxDevices) return EAD_EINVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    StaticDevice &d = g_static_dev[device];
+    if (!d.ready) {
+        int major = 0;
+        EAD_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device));
+        if (major != 10) return EAD_EUNSUPPORTED_ARCH;
+        void *ptr = nullptr;
+        EAD_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        if (!ptr) return EAD_ECUDA;
+        EAD_CUDA(cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, device));
+        EAD_CUDA(cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device));
+        EAD_CUDA(cudaFuncSetAttribute(ead_lmhead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, d.smem_optin));
+        d.scratch = static_cast<StaticScratch *>(ptr);
+        d.ready = true;
+    }
+    *out = &d;
+    return EAD_OK;
+}
+
+}  // namespace
+
+extern "C" int ead_head_entropy_static(const void *W, const void *h, int32_t B, int32_t V, int32_t H, int32_t *tok,
+                                       float *H_out, uint32_t *status, int32_t device, void *stream)
+{
+    if (!W || !h || B < 1 || V < 1 || H < 8) return EAD_EINVALID_ARG;
+    if (B > EAD_STATIC_MAX_B || H > EAD_STATIC_MAX_H) return EAD_ELIMIT;
+    if (H % 8 || !aligned16(W) || !aligned16(h)) return EAD_EALIGNMENT;
+    int ndev = 0;
+    EAD_CUDA(cudaGetDeviceCount(&ndev));
+    if (device < 0 || device >= ndev) return EAD_EINVALID_ARG;
+    EAD_CUDA(cudaSetDevice(device));
+    StaticDevice *d = nullptr;
+    int rc = static_device_setup(device, &d);
+    if (rc != EAD_OK) return rc;
+    StaticScratch *sc = d->scratch;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    const int G = std::min(d->sms, kStaticSlots);
+    const int a_rows = std::min(kTileM, (B + 7) & ~7);
+    const size_t stage_bytes = static_cast<size_t>(a_rows) * kBlockK * 2 + kWTileBytes;
+    const int stages = static_cast<int>(
+        std::min<size_t>(kMaxStages, (static_cast<size_t>(d->smem_optin) - kSmemCtrlBytes - 1024) / stage_bytes));
+    if (stages < 2) return EAD_ECUDA;
+    const size_t smem_bytes = kSmemCtrlBytes + 1024 + stages * stage_bytes;
+
+    // TMA descriptors are built on the host and travel as kernel arguments: no device memory.
+    CUtensorMap tmA, tmW, tmT;
+    const uint32_t wbox = static_cast<uint32_t>(std::min(kTileN, (V + kUnit - 1) / kUnit * kUnit));
+    if (!encode_bf16_2d(&tmA, sc->hidden, kTileM, H, a_rows) || !encode_bf16_2d(&tmW, W, V, H, wbox) ||
+        !encode_bf16_2d(&tmT, W, V, H, kUnit))
+        return EAD_ECUDA;
+
+    ead_static_clear_status_kernel<<<1, 1, 0, s>>>(status);
+    ead_static_stage_kernel<<<a_rows, 128, 0, s>>>(sc, static_cast<const uint16_t *>(h), B, H, a_rows);
+    LmheadParams lp{};
+    lp.V = V;
+    lp.H[0] = H;
+    lp.H[1] = H;
+    lp.a_rows = a_rows;
+    lp.stages = stages;
+    lp.slots_stride = kStaticSlots;
+    lp.B = EAD_STATIC_MAX_B;
+    lp.ctl = &sc->ctl;
+    lp.ctl_rw = &sc->ctl;
+    lp.part_m = sc->part_m;
+    lp.part_s = sc->part_s;
+    lp.part_t = sc->part_t;
+    lp.part_i = sc->part_i;
+    ead_lmhead_kernel<<<G, kLmheadThreads, smem_bytes, s>>>(tmA, tmA, tmW, tmW, tmT, tmT, lp);
+    const int rows_per_block = kGateThreads / 32;
+    ead_static_merge_kernel<<<(B + rows_per_block - 1) / rows_per_block, kGateThreads, 0, s>>>(sc, B, G, tok, H_out,
+                                                                                             status);
+    return cudaGetLastError() == cudaSuccess ? EAD_OK : EAD_ECUDA;
+}
