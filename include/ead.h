@@ -164,6 +164,16 @@ int64_t ead_kernel_launches(const ead_ctx *ctx);
  * box, dynamic shared memory bytes}. */
 int ead_launch_info(const ead_ctx *ctx, int32_t *info, int32_t n);
 
+/*
+ * How the LM-head kernel divides one head among its CTAs (host-side replica of the rule
+ * the kernel applies on the device; pure arithmetic, needs no GPU).  With n rows on a head
+ * there are R = ceil(n / 128) row blocks; CTA `cta` of `G` serves row block out[1] and
+ * vocabulary columns [out[3], out[4]) (multiples of 16; the end may exceed V by < 16).
+ *   out  host, int32 [6]: {active, row_block, slot, col_begin, col_end, group_size}
+ * Errors: EAD_EINVALID_ARG.
+ */
+int ead_plan_split(int32_t cta, int32_t G, int32_t n_rows, int32_t V, int32_t *out);
+
 /* Waits for outstanding work and frees everything the context owns.  NULL is allowed. */
 void ead_destroy(ead_ctx *ctx);
 

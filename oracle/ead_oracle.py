@@ -49,6 +49,10 @@ def lib():
                                         C.c_double, C.c_int32, C.POINTER(C.c_double),
                                         C.POINTER(C.c_uint8), C.POINTER(C.c_uint8),
                                         C.POINTER(C.c_int32)]
+        L.oracle_gate_step.restype = C.c_double
+        L.oracle_gate_step.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int64),
+                                       C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.c_double,
+                                       C.c_int32, C.c_int32, C.c_double]
         L.oracle_run.restype = None
         L.oracle_run.argtypes = ([C.c_int64] * 5 + [C.c_int32, C.c_int32, C.c_double, C.c_int32,
                                                     C.c_int32]
@@ -105,6 +109,22 @@ def gate_trace(H_seq, w: int, d_min: int, tau: float, start_model: int = 0):
                             int(start_model), _p(Hbar, C.c_double), _p(used, C.c_uint8),
                             _p(nxt, C.c_uint8), _p(c_after, C.c_int32))
     return dict(Hbar=Hbar, used=used, next=nxt, c_after=c_after)
+
+
+class GateState:
+    """State of one sequence for step-by-step use of the window / dwell / threshold rule."""
+
+    def __init__(self, capacity: int, start_model: int = 0):
+        self.hist = np.zeros(max(1, capacity), dtype=np.float64)
+        self.n = C.c_int64(0)
+        self.c = C.c_int32(0)
+        self.model = C.c_int32(start_model)
+
+    def step(self, H: float, w: int, d_min: int, tau: float) -> float:
+        """Feeds one entropy; returns the rolling mean; ``self.model.value`` is the next model."""
+        return float(lib().oracle_gate_step(_p(self.hist, C.c_double), C.byref(self.n),
+                                            C.byref(self.c), C.byref(self.model), float(H),
+                                            int(w), int(d_min), float(tau)))
 
 
 def run(W_small, W_large, h_small, h_large, *, w: int, d_min: int, tau: float, unit: int = 0,

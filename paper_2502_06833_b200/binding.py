@@ -28,7 +28,8 @@ EAD_STATUS_BAD_COUNT = 0x4
 
 SYMBOLS = ["ead_create", "ead_step", "ead_run", "ead_run_host", "ead_run_timed", "ead_reset", "ead_status",
            "ead_state_size", "ead_get_state", "ead_set_state", "ead_kernel_launches",
-           "ead_launch_info", "ead_destroy", "ead_strerror", "ead_head_entropy_static"]
+           "ead_launch_info", "ead_destroy", "ead_strerror", "ead_head_entropy_static",
+           "ead_plan_split"]
 
 
 class EadConfig(C.Structure):
@@ -85,6 +86,8 @@ def lib() -> C.CDLL:
         L.ead_head_entropy_static.restype = C.c_int
         L.ead_head_entropy_static.argtypes = [vp, vp, C.c_int32, C.c_int32, C.c_int32, i32p, f32p, vp,
                                               C.c_int32, vp]
+        L.ead_plan_split.restype = C.c_int
+        L.ead_plan_split.argtypes = [C.c_int32] * 4 + [C.POINTER(C.c_int32)]
         L.ead_strerror.restype = C.c_char_p
         L.ead_strerror.argtypes = [C.c_int]
         _lib = L
@@ -195,6 +198,12 @@ def ead_head_entropy_static(W, h, B, V, H, tok=None, H_out=None, status=None, de
     _check(lib().ead_head_entropy_static(_ptr(W), _ptr(h), int(B), int(V), int(H), _ptr(tok),
                                          _ptr(H_out), _ptr(status), int(device),
                                          C.c_void_p(int(stream))), "ead_head_entropy_static")
+
+
+def ead_plan_split(cta, G, n_rows, V) -> dict:
+    a = (C.c_int32 * 6)()
+    _check(lib().ead_plan_split(int(cta), int(G), int(n_rows), int(V), a), "ead_plan_split")
+    return dict(active=a[0], row_block=a[1], slot=a[2], col_begin=a[3], col_end=a[4], group=a[5])
 
 
 def ead_destroy(ctx) -> None:

@@ -316,6 +316,10 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     x->W[0] = W_small;
     x->W[1] = W_large;
     x->G = prop.multiProcessorCount;
+    if ((cfg->B + kTileM - 1) / kTileM > x->G) {   // the work split needs one CTA per row block at least
+        delete x;
+        return EAD_EINVALID_ARG;
+    }
     x->slots_stride = (x->G + 31) & ~31;
     x->a_rows = std::min(kTileM, (cfg->B + 7) & ~7);
     const size_t stage_bytes = static_cast<size_t>(x->a_rows) * kBlockK * 2 + kWTileBytes;
@@ -565,6 +569,20 @@ int ead_launch_info(const ead_ctx *x, int32_t *info, int32_t n)
     if (!x || !info || n < 0) return EAD_EINVALID_ARG;
     const int32_t v[4] = {x->G, x->stages, x->a_rows, static_cast<int32_t>(x->smem_bytes)};
     for (int i = 0; i < n && i < 4; ++i) info[i] = v[i];
+    return EAD_OK;
+}
+
+int ead_plan_split(int32_t cta, int32_t G, int32_t n_rows, int32_t V, int32_t *out)
+{
+    if (!out || cta < 0 || G < 1 || cta >= G || n_rows < 0 || V < 1) return EAD_EINVALID_ARG;
+    if ((n_rows + kTileM - 1) / kTileM > G) return EAD_EINVALID_ARG;   // more row blocks than CTAs
+    const HeadSplit s = split_head(cta, G, n_rows, V);
+    out[0] = s.active;
+    out[1] = s.rb;
+    out[2] = s.slot;
+    out[3] = s.col_begin;
+    out[4] = s.col_end;
+    out[5] = s.g;
     return EAD_OK;
 }
 

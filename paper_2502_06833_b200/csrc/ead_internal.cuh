@@ -64,7 +64,7 @@ __host__ __device__ inline HeadSplit split_head(int cta, int G, int n, int V)
         return s;
     }
     s.g = G / s.R;
-    if (s.g < 1) s.g = 1;      // only if R > G; then CTAs take several row blocks (not used: B <= 4096)
+    if (s.g < 1) s.g = 1;      // R > G is rejected on the host (B <= 4096 gives R <= 32)
     s.active = cta < s.g * s.R;
     s.rb = cta % s.R;
     s.slot = cta / s.R;

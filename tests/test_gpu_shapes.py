@@ -1,0 +1,199 @@
+"""Parity with the oracle on small shapes that span several tiles, ragged tails, several
+row blocks and both heads in one step; and the properties that hold at any size."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import ead_oracle as O
+from workloads import synth
+from workloads.configs import EADConfig
+
+from gpu_util import GpuGate, compare
+
+pytestmark = pytest.mark.gpu
+
+
+def _cfg(**kw):
+    base = dict(name="case", B=4, T=24, H_small=64, H_large=128, V=1000, tau=5.2, w=3, d_min=2,
+                seed=7, stay_easy=0.8, stay_hard=0.8)
+    base.update(kw)
+    return EADConfig(**base)
+
+
+def _oracle(cfg, wl, rows=None, T=None):
+    return O.run(wl.W_small, wl.W_large, wl.h_small, wl.h_large, w=cfg.w, d_min=cfg.d_min,
+                 tau=float(np.float32(cfg.tau)), unit=cfg.unit, start_model=cfg.start_model,
+                 rows=rows, T=T)
+
+
+def _mid_tau(V):
+    """A threshold between the entropy modes of the generator for vocabulary size V."""
+    return 0.5 * (math.log(V) + (math.log(V) - 4.5))
+
+
+SHAPES = [
+    # B, V, H_small, H_large        what it exercises
+    (1, 1000, 64, 128),           # single row, V not a multiple of 16
+    (3, 257, 72, 200),            # tiny ragged V, hidden sizes that are not multiples of 64
+    (5, 4100, 256, 512),          # ragged tail after full 256-wide tiles
+    (37, 16, 8, 16),              # fewer vocabulary units than CTAs, smallest hidden sizes
+    (8, 40000, 128, 64),          # several 256-wide tiles per CTA; large head narrower than small
+    (130, 3000, 64, 128),         # two row blocks, the second with 2 rows
+    (300, 5000, 128, 256),        # three row blocks shared by both heads
+    (128, 2048, 64, 64),          # exactly one full row block
+]
+
+
+@pytest.mark.parametrize("B,V,Hs,Hl", SHAPES)
+def test_small_shapes_full_parity(B, V, Hs, Hl):
+    cfg = _cfg(B=B, V=V, H_small=Hs, H_large=Hl, tau=_mid_tau(V), T=20 if B > 64 else 28)
+    wl = synth.Workload(cfg)
+    ora = _oracle(cfg, wl)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        out = g.run(wl.h_small, wl.h_large, "run")
+    log = compare(out, ora, cfg.tau)
+    assert log["cells"] >= 0.9 * cfg.B * cfg.T
+    if V > 16:
+        assert 0.02 < out["used"].mean() < 0.98, "the case should exercise both heads"
+
+
+@pytest.mark.parametrize("w,d_min,start", [(1, 1, 0), (1, 0, 1), (20, 10, 0), (5, 3, 1), (64, 1, 0)])
+def test_window_and_dwell_variants(w, d_min, start):
+    cfg = _cfg(B=6, V=1500, T=48, w=w, d_min=d_min, start_model=start, tau=_mid_tau(1500))
+    wl = synth.Workload(cfg)
+    ora = _oracle(cfg, wl)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        out = g.run(wl.h_small, wl.h_large, "run")
+    compare(out, ora, cfg.tau)
+
+
+def test_bits_convention_gives_the_nats_switch_trace():
+    cfg = _cfg(B=5, V=2000, T=40, tau=_mid_tau(2000))
+    wl = synth.Workload(cfg)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        nats = g.run(wl.h_small, wl.h_large, "run")
+    cfg_b = cfg.with_(unit=1, tau=cfg.tau / math.log(2.0))
+    ora_b = _oracle(cfg_b, wl)
+    with GpuGate(cfg_b, wl.W_small, wl.W_large) as g:
+        bits = g.run(wl.h_small, wl.h_large, "run")
+    compare(bits, ora_b, cfg_b.tau, unit=1)
+    assert np.array_equal(bits["used"], nats["used"]) and np.array_equal(bits["tok"], nats["tok"])
+    np.testing.assert_allclose(bits["H"], nats["H"] / math.log(2.0), rtol=2e-6)
+
+
+def test_step_run_and_host_entry_points_agree_bit_for_bit():
+    cfg = _cfg(B=9, V=3000, T=70, tau=_mid_tau(3000))        # 70 = 2 graph chunks of 32 + 6 single steps
+    wl = synth.Workload(cfg)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        a = g.run(wl.h_small, wl.h_large, "run")
+        g.E.ead_reset(g.ctx)
+        b = g.run(wl.h_small, wl.h_large, "step")
+        g.E.ead_reset(g.ctx)
+        c = g.run(wl.h_small, wl.h_large, "host")
+        g.E.ead_reset(g.ctx)
+        d1 = g.run(wl.h_small[:33], wl.h_large[:33], "run")      # a run continues where the last ended
+        d2 = g.run(wl.h_small[33:], wl.h_large[33:], "run")
+    for k in ("tok", "H", "Hbar", "used", "next"):
+        assert np.array_equal(a[k], b[k]), k
+        assert np.array_equal(a[k], c[k]), k
+        assert np.array_equal(a[k], np.concatenate([d1[k], d2[k]])), k
+    assert 0.05 < a["used"].mean() < 0.95
+
+
+def test_checkpoint_and_resume():
+    cfg = _cfg(B=7, V=1200, T=40, tau=_mid_tau(1200))
+    wl = synth.Workload(cfg)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        full = g.run(wl.h_small, wl.h_large, "run")
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        g.run(wl.h_small[:17], wl.h_large[:17], "run")
+        blob = g.E.ead_get_state(g.ctx)
+        assert len(blob) == g.E.ead_state_size(g.ctx)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        g.E.ead_set_state(g.ctx, blob)
+        rest = g.run(wl.h_small[17:], wl.h_large[17:], "run")
+        with pytest.raises(g.E.EadError) as err:
+            g.E.ead_set_state(g.ctx, blob[:-4])
+        assert err.value.code == g.E.EAD_ESTATE
+    for k in ("tok", "H", "Hbar", "used", "next"):
+        assert np.array_equal(full[k][17:], rest[k]), k
+
+
+def test_rows_are_independent_and_permutation_equivariant():
+    cfg = _cfg(B=12, V=2500, T=30, tau=_mid_tau(2500))
+    wl = synth.Workload(cfg)
+    perm = np.random.default_rng(3).permutation(cfg.B)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        a = g.run(wl.h_small, wl.h_large, "run")
+        g.E.ead_reset(g.ctx)
+        b = g.run(wl.h_small[:, perm], wl.h_large[:, perm], "run")
+    for k in ("tok", "used", "next"):
+        assert np.array_equal(a[k][:, perm], b[k]), k
+    # the compacted position of a row changes with the batch around it, the arithmetic per row does not
+    np.testing.assert_array_equal(a["H"][:, perm], b["H"])
+    sub = cfg.with_(B=5)
+    with GpuGate(sub, wl.W_small, wl.W_large) as g:
+        c = g.run(wl.h_small[:, :5], wl.h_large[:, :5], "run")
+    assert np.array_equal(c["tok"], a["tok"][:, :5]) and np.array_equal(c["used"], a["used"][:, :5])
+    np.testing.assert_allclose(c["H"], a["H"][:, :5], atol=1e-5)
+
+
+def test_non_finite_hidden_state_is_reported_and_leaves_the_row_untouched():
+    cfg = _cfg(B=4, V=900, T=12, tau=_mid_tau(900))
+    wl = synth.Workload(cfg)
+    hs, hl = wl.h_small.copy(), wl.h_large.copy()
+    hs[5, 2, 3] = 0x7FC0            # bf16 NaN in row 2 at step 5 (both models, whichever is active)
+    hl[5, 2, 3] = 0x7FC0
+    hs[7, 1, 0] = 0x7F80            # +inf in row 1 at step 7
+    hl[7, 1, 0] = 0x7F80
+    ora = O.run(wl.W_small, wl.W_large, hs, hl, w=cfg.w, d_min=cfg.d_min,
+                tau=float(np.float32(cfg.tau)))
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        E = g.E
+        from gpu_util import to_dev_bf16
+        import torch
+        d_hs, d_hl = to_dev_bf16(hs), to_dev_bf16(hl)
+        o = g._outs(cfg.T)
+        E.ead_run(g.ctx, cfg.T, d_hs, d_hl, o["tok"], o["H"], o["Hbar"], o["used"], o["next"])
+        word = E.ead_status(g.ctx)
+        out = g._np(o)
+    assert word == E.EAD_STATUS_NONFINITE
+    for (t, b) in ((5, 2), (7, 1)):
+        assert math.isnan(out["H"][t, b]) and math.isnan(out["Hbar"][t, b]) and out["tok"][t, b] == -1
+        assert math.isnan(ora["H"][t, b]) and ora["tok"][t, b] == -1
+        assert out["used"][t, b] == out["next"][t, b] == ora["used"][t, b]
+    ok = np.isfinite(ora["H"])
+    assert np.array_equal(np.isfinite(out["H"]), ok)
+    assert np.array_equal(out["tok"], ora["tok"]) and np.array_equal(out["used"], ora["used"])
+    assert np.array_equal(out["next"], ora["next"])
+    np.testing.assert_allclose(out["H"][ok], ora["H"][ok], atol=2e-3)
+    np.testing.assert_allclose(out["Hbar"][ok], ora["Hbar"][ok], atol=2e-3)
+
+
+def test_closed_forms_on_the_gpu():
+    """Uniform logits (zero hidden state) give ln V; a one-hot-like row gives ~0 and its index."""
+    V, H = 3000, 64
+    cfg = _cfg(B=2, V=V, H_small=H, H_large=H, T=1, tau=99.0)
+    W = np.zeros((V, H), dtype=np.float32)
+    W[:, 0] = 0.0
+    W[1234, 1] = 8.0
+    Wb = synth.f32_to_bf16_bits(W)
+    h = np.zeros((1, 2, H), dtype=np.float32)
+    h[0, 1, 1] = 8.0                                   # row 1: logit 64 at column 1234, 0 elsewhere
+    hb = synth.f32_to_bf16_bits(h)
+    with GpuGate(cfg, Wb, Wb) as g:
+        out = g.run(hb, hb, "run")
+    assert out["H"][0, 0] == pytest.approx(math.log(V), abs=1e-5)
+    assert out["tok"][0, 0] == 0                       # all equal: lowest index
+    assert 0.0 <= out["H"][0, 1] < 1e-6 and out["tok"][0, 1] == 1234
+
+
+def test_largest_batch_and_zero_steps():
+    cfg = _cfg(B=1024, V=600, H_small=16, H_large=8, T=4, tau=_mid_tau(600), d_min=1, w=1)
+    wl = synth.Workload(cfg)
+    ora = _oracle(cfg, wl)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        g.E.ead_run(g.ctx, 0, 16, 16)                  # T = 0 is a no-op
+        out = g.run(wl.h_small, wl.h_large, "run")
+    compare(out, ora, cfg.tau)

@@ -1,0 +1,145 @@
+"""CPU-only checks of the host side: the C-ABI library loads and exports what
+include/ead.h declares, argument validation, the CTA work split, bench helpers and the
+multi-process aggregation (gloo, world size 2)."""
+import os
+import re
+import subprocess
+import sys
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def E():
+    from paper_2502_06833_b200 import build
+    build.build()
+    from paper_2502_06833_b200 import binding
+    return binding
+
+
+def test_library_exports_every_declared_symbol(E):
+    hdr = open(os.path.join(ROOT, "include", "ead.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = set(re.findall(r"\b(ead_[a-z_]+)\s*\(", hdr))
+    assert declared, "no declarations found"
+    lib = E.lib()
+    for name in sorted(declared):
+        assert hasattr(lib, name), f"{name} is declared but not exported"
+    assert declared == set(E.SYMBOLS)
+
+
+def test_strerror_names_every_code(E):
+    for code in range(0, -8, -1):
+        assert E.strerror(code) != "unknown error"
+    assert E.strerror(-99) == "unknown error"
+
+
+def test_create_rejects_bad_arguments_before_touching_the_gpu(E):
+    good = dict(B=4, V=100, H_small=64, H_large=128, w=5, d_min=10, tau=2.0, W_small=4096,
+                W_large=8192)
+    for bad, code in [(dict(B=0), E.EAD_EINVALID_ARG), (dict(B=5000), E.EAD_EINVALID_ARG),
+                      (dict(V=0), E.EAD_EINVALID_ARG), (dict(w=0), E.EAD_EINVALID_ARG),
+                      (dict(w=65), E.EAD_EINVALID_ARG), (dict(unit=2), E.EAD_EINVALID_ARG),
+                      (dict(start_model=3), E.EAD_EINVALID_ARG),
+                      (dict(W_small=None), E.EAD_EINVALID_ARG),
+                      (dict(H_small=60), E.EAD_EALIGNMENT), (dict(H_large=4), E.EAD_EINVALID_ARG),
+                      (dict(W_large=8200), E.EAD_EALIGNMENT)]:
+        with pytest.raises(E.EadError) as err:
+            E.ead_create(**{**good, **bad})
+        assert err.value.code == code, (bad, err.value.code)
+
+
+def test_null_context_is_an_error_not_a_crash(E):
+    for fn, args in [(E.ead_reset, (None,)), (E.ead_step, (None, 16, 16)),
+                     (E.ead_run, (None, 1, 16, 16))]:
+        with pytest.raises(E.EadError) as err:
+            fn(*args)
+        assert err.value.code == E.EAD_EINVALID_ARG
+    E.ead_destroy(None)
+    assert E.lib().ead_state_size(None) == 0
+
+
+def test_static_entry_point_limits_are_checked_on_the_host(E):
+    with pytest.raises(E.EadError) as err:
+        E.ead_head_entropy_static(4096, 8192, E.EAD_STATIC_MAX_B + 1, 100, 64)
+    assert err.value.code == E.EAD_ELIMIT
+    with pytest.raises(E.EadError) as err:
+        E.ead_head_entropy_static(4096, 8192, 4, 100, 60)
+    assert err.value.code == E.EAD_EALIGNMENT
+
+
+@pytest.mark.parametrize("G,n,V", [(148, 1, 128256), (148, 64, 128256), (148, 192, 152064),
+                                   (148, 1024, 152064), (148, 4096, 1000), (148, 5, 37),
+                                   (148, 129, 4100), (132, 300, 5000), (8, 1000, 257)])
+def test_work_split_covers_every_column_once_per_row_block(E, G, n, V):
+    R = (n + 127) // 128
+    cover = np.zeros((R, (V + 15) // 16 * 16), dtype=np.int32)
+    spans, slots = [], {}
+    for cta in range(G):
+        s = E.ead_plan_split(cta, G, n, V)
+        if not s["active"]:
+            assert s["col_begin"] == s["col_end"]
+            continue
+        assert s["col_begin"] % 16 == 0 and s["col_end"] % 16 == 0
+        assert 0 <= s["row_block"] < R and 0 <= s["slot"] < s["group"] <= 160
+        cover[s["row_block"], s["col_begin"]:s["col_end"]] += 1
+        spans.append(s["col_end"] - s["col_begin"])
+        assert slots.setdefault((s["row_block"], s["slot"]), cta) == cta
+    assert (cover == 1).all(), "a column is missed or served twice"
+    assert max(spans) - min(spans) <= 16          # balanced to one 16-column unit
+    assert len(slots) == R * max(1, G // R)
+
+
+def test_work_split_needs_a_cta_per_row_block(E):
+    with pytest.raises(E.EadError) as err:
+        E.ead_plan_split(0, 4, 1000, 257)
+    assert err.value.code == E.EAD_EINVALID_ARG
+
+
+def test_work_split_of_an_empty_head(E):
+    s = E.ead_plan_split(0, 148, 0, 1000)
+    assert s["active"] == 0 and s["col_begin"] == s["col_end"]
+
+
+def test_bench_step_costs():
+    sys.path.insert(0, ROOT)
+    import bench
+    from workloads import configs
+    cfg = configs.LLAMA_B64
+    used = np.zeros((3, cfg.B), dtype=np.uint8)
+    used[1, :10] = 1
+    used[2, :] = 1
+    b, f = bench.step_costs(cfg, used)
+    ws, wl = 2 * cfg.V * cfg.H_small, 2 * cfg.V * cfg.H_large
+    assert b[0] == ws + 2 * 64 * cfg.H_small
+    assert b[1] == ws + wl + 2 * (54 * cfg.H_small + 10 * cfg.H_large)
+    assert b[2] == wl + 2 * 64 * cfg.H_large
+    assert f[1] == 2 * cfg.V * (54 * cfg.H_small + 10 * cfg.H_large)
+
+
+_GLOO_WORKER = r"""
+import os, sys
+sys.path.insert(0, {root!r})
+import torch.distributed as dist
+import bench
+dist.init_process_group("gloo")
+rank = dist.get_rank()
+value, t, world = bench.aggregate_over_ranks(10.0 * (rank + 1), 100, dist)
+assert world == 2 and abs(t - 20.0) < 1e-9 and abs(value - 2 * 100 / 0.020) < 1e-6, (value, t, world)
+dist.barrier()
+dist.destroy_process_group()
+print("rank", rank, "ok")
+"""
+
+
+def test_aggregation_over_two_ranks_takes_the_slowest(tmp_path):
+    script = tmp_path / "worker.py"
+    script.write_text(_GLOO_WORKER.format(root=ROOT))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+           "--master-addr", "127.0.0.1", "--master-port", "29631", str(script)]
+    res = subprocess.run(cmd, capture_output=True, text=True, timeout=240)
+    assert res.returncode == 0, res.stdout + res.stderr
+    assert res.stdout.count("ok") == 2
