@@ -15,6 +15,7 @@
 #include "ead_internal.cuh"
 #include "gate_kernels.cuh"
 #include "lmhead_kernel.cuh"
+#include "lmhead_small_kernel.cuh"
 
 using namespace ead;
 
@@ -69,6 +70,7 @@ struct ead_ctx {
     cudaStream_t stream = nullptr;
     cudaStream_t cap_stream = nullptr;     // capture happens on a private stream
     int G = 0, a_rows = 0, stages = 0, slots_stride = 0;
+    int small_cols = 0;                    // > 0: swapped-operand kernel with this many batch columns
     size_t smem_bytes = 0;
     const void *W[2] = {nullptr, nullptr};
     // device state and scratch (owned)
@@ -117,6 +119,7 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     lp.H[0] = c.H_small;
     lp.H[1] = c.H_large;
     lp.a_rows = x->a_rows;
+    lp.n_cols = x->small_cols;
     lp.stages = x->stages;
     lp.slots_stride = x->slots_stride;
     lp.B = c.B;
@@ -126,8 +129,18 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     lp.part_s = x->part_s;
     lp.part_t = x->part_t;
     lp.part_i = x->part_i;
-    ead_lmhead_kernel<<<x->G, kLmheadThreads, x->smem_bytes, s>>>(x->tmA[0], x->tmA[1], x->tmW[0], x->tmW[1],
-                                                                  x->tmT[0], x->tmT[1], lp);
+#define EAD_LAUNCH_LMHEAD(kernel)                                                                              \
+    kernel<<<x->G, kLmheadThreads, x->smem_bytes, s>>>(x->tmA[0], x->tmA[1], x->tmW[0], x->tmW[1], x->tmT[0], \
+                                                       x->tmT[1], lp)
+    switch (x->small_cols) {
+        case 0: EAD_LAUNCH_LMHEAD(ead_lmhead_kernel); break;
+        case 1: EAD_LAUNCH_LMHEAD(ead_lmhead_small_kernel<1>); break;
+        case 2: EAD_LAUNCH_LMHEAD(ead_lmhead_small_kernel<2>); break;
+        case 4: EAD_LAUNCH_LMHEAD(ead_lmhead_small_kernel<4>); break;
+        case 8: EAD_LAUNCH_LMHEAD(ead_lmhead_small_kernel<8>); break;
+        default: EAD_LAUNCH_LMHEAD(ead_lmhead_small_kernel<16>); break;
+    }
+#undef EAD_LAUNCH_LMHEAD
     if (ev) cudaEventRecord(ev[2], s);
 
     GateParams gp{};
@@ -321,9 +334,18 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
         return EAD_EINVALID_ARG;
     }
     x->slots_stride = (x->G + 31) & ~31;
-    x->a_rows = std::min(kTileM, (cfg->B + 7) & ~7);
-    const size_t stage_bytes = static_cast<size_t>(x->a_rows) * kBlockK * 2 + kWTileBytes;
     const size_t smem_max = prop.sharedMemPerBlockOptin;
+    size_t stage_bytes;
+    if (cfg->B <= kSmallN) {
+        // latency regime: swapped-operand kernel, batch columns rounded up to a power of two
+        x->small_cols = 1;
+        while (x->small_cols < cfg->B) x->small_cols *= 2;
+        x->a_rows = kSmallN;
+        stage_bytes = kSmallStageBytes;
+    } else {
+        x->a_rows = std::min(kTileM, (cfg->B + 7) & ~7);
+        stage_bytes = static_cast<size_t>(x->a_rows) * kBlockK * 2 + kWTileBytes;
+    }
     x->stages = static_cast<int>(std::min<size_t>(kMaxStages, (smem_max - kSmemCtrlBytes - 1024) / stage_bytes));
     x->smem_bytes = kSmemCtrlBytes + 1024 + x->stages * stage_bytes;
 
@@ -358,7 +380,8 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     cudaMemsetAsync(x->part_t, 0, 4 * np, x->stream);
     cudaMemsetAsync(x->part_i, 0, 4 * np, x->stream);
 
-    const uint32_t wbox = static_cast<uint32_t>(std::min(kTileN, (cfg->V + kUnit - 1) / kUnit * kUnit));
+    const uint32_t wbox = static_cast<uint32_t>(
+        std::min(x->small_cols ? kSmallTileRows : kTileN, (cfg->V + kUnit - 1) / kUnit * kUnit));
     const int Hm[2] = {cfg->H_small, cfg->H_large};
     for (int m = 0; m < 2; ++m) {
         if (!encode_bf16_2d(&x->tmA[m], x->hc[m], Bpad, Hm[m], x->a_rows) ||
@@ -368,9 +391,19 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     }
     // the attribute belongs to the kernel on this device, not to the context: ask for the
     // device maximum so that contexts with different stage counts can coexist
-    if (cudaFuncSetAttribute(ead_lmhead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(smem_max)) != cudaSuccess)
-        return fail(EAD_ECUDA);
+    const void *lmhead_kernels[] = {
+        reinterpret_cast<const void *>(ead_lmhead_kernel),          reinterpret_cast<const void *>(ead_lmhead_small_kernel<1>),
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<2>), reinterpret_cast<const void *>(ead_lmhead_small_kernel<4>),
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<8>), reinterpret_cast<const void *>(ead_lmhead_small_kernel<16>)};
+    for (const void *k : lmhead_kernels) {
+        cudaFuncAttributes fa;
+        if (cudaFuncGetAttributes(&fa, k) != cudaSuccess) return fail(EAD_ECUDA);
+        const size_t dyn_max = smem_max - fa.sharedSizeBytes;      // static shared memory counts too
+        if (x->smem_bytes > dyn_max) return fail(EAD_ECUDA);
+        if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(dyn_max)) !=
+            cudaSuccess)
+            return fail(EAD_ECUDA);
+    }
     if (cudaFuncSetAttribute(ead_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * 4096) !=
         cudaSuccess)
         return fail(EAD_ECUDA);

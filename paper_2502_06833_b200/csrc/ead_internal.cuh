@@ -75,10 +75,35 @@ __host__ __device__ inline HeadSplit split_head(int cta, int G, int n, int V)
     return s;
 }
 
+#ifdef __CUDACC__
+struct Partial {
+    float m, s, t;
+    int idx;
+};
+
+// Combines the statistics of two disjoint column sets (m = max z, s = sum exp(z - m),
+// t = sum exp(z - m) (z - m) log2 e, idx = lowest column attaining m).  Equal maxima keep the lower column.
+__device__ __forceinline__ Partial merge_partial(const Partial &a, const Partial &b)
+{
+    Partial r;
+    r.m = fmaxf(a.m, b.m);
+    const float da = (a.m - r.m) * kLog2e, db = (b.m - r.m) * kLog2e;
+    const float ea = exp2f(da), eb = exp2f(db);
+    r.s = ea * a.s + eb * b.s;
+    r.t = ea * fmaf(da, a.s, a.t) + eb * fmaf(db, b.s, b.t);
+    if (a.m > b.m) r.idx = a.idx;
+    else if (b.m > a.m) r.idx = b.idx;
+    else r.idx = min(a.idx, b.idx);
+    return r;
+}
+
+#endif  // __CUDACC__
+
 struct LmheadParams {
     int32_t V;
     int32_t H[2];
     int32_t a_rows;        // rows of the hidden-state TMA box (multiple of 8, <= 128)
+    int32_t n_cols;        // small-batch kernel: batch columns kept per thread (power of two <= 16)
     int32_t stages;
     int32_t slots_stride;  // partial slots per row (>= CTAs)
     int32_t B;

@@ -96,27 +96,6 @@ ead_compact_kernel(StepCtl *ctl, const RunArgs *args, const uint8_t *flag, int B
     }
 }
 
-struct Partial {
-    float m, s, t;
-    int idx;
-};
-
-// Combines the statistics of two disjoint column sets (see lmhead_kernel.cuh for the
-// meaning of m, s, t).  Equal maxima keep the lower column.
-__device__ __forceinline__ Partial merge_partial(const Partial &a, const Partial &b)
-{
-    Partial r;
-    r.m = fmaxf(a.m, b.m);
-    const float da = (a.m - r.m) * kLog2e, db = (b.m - r.m) * kLog2e;
-    const float ea = exp2f(da), eb = exp2f(db);
-    r.s = ea * a.s + eb * b.s;
-    r.t = ea * fmaf(da, a.s, a.t) + eb * fmaf(db, b.s, b.t);
-    if (a.m > b.m) r.idx = a.idx;
-    else if (b.m > a.m) r.idx = b.idx;
-    else r.idx = min(a.idx, b.idx);
-    return r;
-}
-
 struct GateParams {
     int32_t B, V, w, d_min, unit, G, slots_stride;
     float tau;

@@ -1,0 +1,251 @@
+// LM-head projection + online entropy / arg-max statistics for SMALL batches (B <= 16).
+//
+// At a handful of sequences the step is bound by streaming the weights from HBM, and an
+// MMA with the batch on the M side would spend 128 tensor-core rows on 1-16 real ones.
+// This kernel swaps the operands instead: MMA M (TMEM lanes) = 128 vocabulary rows of W,
+// MMA N (TMEM columns) = 16 batch columns, K = hidden, so the tensor work is 16x smaller
+// and W is the only operand of any size.  One epilogue thread owns one vocabulary row of
+// every tile (rows r, r + 128, ... of the CTA's range) and keeps NB running statistics,
+// one per sequence; they are merged across the 128 threads once, at the end of the range.
+// The result is written in the same per-CTA partial format as ead_lmhead_kernel, so the
+// merge + gate kernel does not care which of the two produced it.
+//
+// Pipeline: per K block of 128 hidden elements one stage = two 64-wide W boxes (128 rows
+// each, 16 KiB) + two 64-wide boxes of the compacted hidden rows (16 rows, 2 KiB); TMEM
+// holds two 16-column accumulators so that the epilogue overlaps the next tile's MMAs.
+#pragma once
+#include "lmhead_kernel.cuh"
+
+namespace ead {
+
+constexpr int kSmallTileRows = 128;                    // vocabulary rows per tile (MMA M)
+constexpr int kSmallN = 16;                            // batch columns (MMA N)
+constexpr int kSmallBlockK = 128;                      // hidden elements per stage
+constexpr int kSmallHBytes = kSmallN * 64 * 2;         // one 64-wide box of hidden rows: 2 KiB
+constexpr int kSmallWBytes = kSmallTileRows * 64 * 2;  // one 64-wide box of W rows: 16 KiB
+constexpr int kSmallStageBytes = 2 * kSmallHBytes + 2 * kSmallWBytes;   // 36 KiB
+constexpr int kSmallTmemCols = 32;                     // 2 accumulators x 16 columns
+
+template <int NB>
+__global__ void __launch_bounds__(kLmheadThreads, 1)
+ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
+                        const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
+                        const __grid_constant__ CUtensorMap tmT0, const __grid_constant__ CUtensorMap tmT1,
+                        const LmheadParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                                ~static_cast<uintptr_t>(1023));
+    SmemCtrl *ctrl = reinterpret_cast<SmemCtrl *>(smem);
+    uint8_t *stage0 = smem + kSmemCtrlBytes;
+    __shared__ Partial xwarp[4][NB];
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int cta = blockIdx.x;
+    const int G = gridDim.x;
+    const int stages = p.stages;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < stages; ++i) {
+            mbar_init(smem_u32(&ctrl->full[i]), 1);
+            mbar_init(smem_u32(&ctrl->empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&ctrl->tmem_full[i]), 1);
+            mbar_init(smem_u32(&ctrl->tmem_empty[i]), 4);
+        }
+        mbar_init(smem_u32(&ctrl->drain), 1);
+        ctrl->abort = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0 && lane == 0) {
+        tma_prefetch_desc(&tmA0); tma_prefetch_desc(&tmA1);
+        tma_prefetch_desc(&tmW0); tma_prefetch_desc(&tmW1);
+        tma_prefetch_desc(&tmT0); tma_prefetch_desc(&tmT1);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&ctrl->tmem_base), kSmallTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&ctrl->tmem_base);
+
+    const int n_rows[2] = {p.ctl->n[0], p.ctl->n[1]};
+    StepCtl *ctl = p.ctl_rw;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            const uint64_t pol_keep = l2_policy_evict_last();
+            uint32_t it = 0;
+            bool ok = true;
+            for (int m = 0; m < 2 && ok; ++m) {
+                const HeadSplit sp = split_head(cta, G, n_rows[m], p.V);   // n <= 16: one row block
+                if (!sp.active) continue;
+                const CUtensorMap *tA = m ? &tmA1 : &tmA0;
+                const CUtensorMap *tW = m ? &tmW1 : &tmW0;
+                const CUtensorMap *tT = m ? &tmT1 : &tmT0;
+                const int kblocks = (p.H[m] + kSmallBlockK - 1) / kSmallBlockK;
+                for (int row0 = sp.col_begin; row0 < sp.col_end && ok; row0 += kSmallTileRows) {
+                    const int nrows = min(kSmallTileRows, sp.col_end - row0);
+                    const uint32_t tx = 2 * kSmallHBytes + 2 * static_cast<uint32_t>(nrows) * 128;
+                    for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                        const uint32_t s = it % stages;
+                        const uint32_t ph = (it / stages) & 1u;
+                        if (!wait_bar(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, ctl)) { ok = false; break; }
+                        const uint32_t bar = smem_u32(&ctrl->full[s]);
+                        const uint32_t sa = smem_u32(stage0 + static_cast<size_t>(s) * kSmallStageBytes);
+                        mbar_arrive_expect_tx(bar, tx);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const int k0 = kb * kSmallBlockK + h * 64;
+                            tma_load_2d(sa + h * kSmallHBytes, tA, k0, 0, bar, pol_keep);
+                            const uint32_t wdst = sa + 2 * kSmallHBytes + h * kSmallWBytes;
+                            if (nrows == kSmallTileRows) {
+                                tma_load_2d(wdst, tW, k0, row0, bar, pol_keep);
+                            } else {
+                                for (int j = 0; j < nrows; j += kUnit)
+                                    tma_load_2d(wdst + j * 128, tT, k0, row0 + j, bar, pol_keep);
+                            }
+                        }
+                    }
+                }
+            }
+            const uint32_t pending = it < static_cast<uint32_t>(stages) ? it : stages;
+            for (uint32_t k = 0; k < pending; ++k) {
+                const uint32_t j = it - 1 - k;
+                if (!wait_bar(smem_u32(&ctrl->full[j % stages]), (j / stages) & 1u, ctrl, ctl)) break;
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            uint32_t it = 0, tc = 0;
+            bool ok = true;
+            const uint32_t idesc = umma_idesc_bf16_m128(kSmallN);
+            for (int m = 0; m < 2 && ok; ++m) {
+                const HeadSplit sp = split_head(cta, G, n_rows[m], p.V);
+                if (!sp.active) continue;
+                const int kblocks = (p.H[m] + kSmallBlockK - 1) / kSmallBlockK;
+                for (int row0 = sp.col_begin; row0 < sp.col_end && ok; row0 += kSmallTileRows, ++tc) {
+                    const uint32_t buf = tc & 1u;
+                    if (!wait_bar(smem_u32(&ctrl->tmem_empty[buf]), ((tc >> 1) & 1u) ^ 1u, ctrl, ctl)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint32_t d_tmem = tmem_base + buf * kSmallN;
+                    for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                        const uint32_t s = it % stages;
+                        if (!wait_bar(smem_u32(&ctrl->full[s]), (it / stages) & 1u, ctrl, ctl)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after_sync();
+                        const uint32_t sa = smem_u32(stage0 + static_cast<size_t>(s) * kSmallStageBytes);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint64_t dh = umma_smem_desc(sa + h * kSmallHBytes);                      // B: hidden rows
+                            const uint64_t dw = umma_smem_desc(sa + 2 * kSmallHBytes + h * kSmallWBytes);   // A: W rows
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                umma_bf16(d_tmem, dw + 2 * k, dh + 2 * k, idesc, (kb | h | k) != 0);
+                        }
+                        umma_commit(smem_u32(&ctrl->empty[s]));
+                    }
+                    if (ok) umma_commit(smem_u32(&ctrl->tmem_full[buf]));
+                }
+            }
+            umma_commit(smem_u32(&ctrl->drain));
+            wait_bar(smem_u32(&ctrl->drain), 0u, ctrl, ctl);
+        }
+    } else {
+        // ------------------------------------------------------------- epilogue
+        const int quad = warp & 3;
+        const int ew = warp - 2;                       // 0..3
+        uint32_t tc = 0;
+        bool ok = true;
+        // Every epilogue warp passes the same named barriers whatever happened to its waits,
+        // so a warp that gave up cannot leave the others stuck at one.
+        for (int m = 0; m < 2; ++m) {
+            const HeadSplit sp = split_head(cta, G, n_rows[m], p.V);
+            if (!sp.active) continue;
+            float sm[NB], ss[NB], stt[NB];
+            int sidx[NB];
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                sm[j] = kNegSentinel;
+                ss[j] = 0.f;
+                stt[j] = 0.f;
+                sidx[j] = 0x7fffffff;
+            }
+            const int row_limit = min(p.V, sp.col_end);
+            for (int row0 = sp.col_begin; row0 < sp.col_end && ok; row0 += kSmallTileRows, ++tc) {
+                const uint32_t buf = tc & 1u;
+                if (!wait_bar_warp(smem_u32(&ctrl->tmem_full[buf]), (tc >> 1) & 1u, ctrl, ctl, lane)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after_sync();
+                float v[16];
+                tmem_ld_16cols(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + buf * kSmallN, v);
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[buf]));
+                const int row = row0 + quad * 32 + lane;          // vocabulary entry of this thread
+                if (row < row_limit) {
+#pragma unroll
+                    for (int j = 0; j < NB; ++j) {
+                        const float z = v[j];
+                        const float mo = sm[j];
+                        const float mn = fmaxf(mo, z);
+                        const float dm2 = (mo - mn) * kLog2e;       // <= 0
+                        const float dz2 = (z - mn) * kLog2e;        // <= 0
+                        const float a = ex2_approx(dm2), e = ex2_approx(dz2);
+                        stt[j] = fmaf(a, fmaf(dm2, ss[j], stt[j]), e * dz2);
+                        ss[j] = fmaf(a, ss[j], e);
+                        sidx[j] = (z > mo) ? row : sidx[j];
+                        sm[j] = mn;
+                    }
+                }
+                __syncwarp();
+            }
+            // ---- merge the 128 per-thread statistics of every sequence: lanes, then warps
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                Partial acc{sm[j], ss[j], stt[j], sidx[j]};
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    Partial q;
+                    q.m = __shfl_xor_sync(0xffffffffu, acc.m, o);
+                    q.s = __shfl_xor_sync(0xffffffffu, acc.s, o);
+                    q.t = __shfl_xor_sync(0xffffffffu, acc.t, o);
+                    q.idx = __shfl_xor_sync(0xffffffffu, acc.idx, o);
+                    acc = merge_partial(acc, q);
+                }
+                if (lane == 0) xwarp[ew][j] = acc;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");        // the four epilogue warps only
+            if (ew == 0 && lane < NB && lane < n_rows[m] && ok) {
+                Partial acc = xwarp[0][lane];
+                for (int k = 1; k < 4; ++k) acc = merge_partial(acc, xwarp[k][lane]);
+                const size_t o = (static_cast<size_t>(m) * p.B + lane) * p.slots_stride + sp.slot;
+                p.part_m[o] = acc.m;
+                p.part_s[o] = acc.s;
+                p.part_t[o] = acc.t;
+                p.part_i[o] = acc.idx;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");        // xwarp is reused by the next head
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 1) tmem_dealloc(tmem_base, kSmallTmemCols);
+}
+
+}  // namespace ead

@@ -1,0 +1,69 @@
+"""Full-size configurations, in the launch configuration the benchmark times, against
+stored oracle results (tests/golden/oracle_*.npz, written by tests/golden/make_golden.py,
+which calls only the oracle).  The GPU runs the whole batch for the whole T; compared are
+all rows over the first steps and a few rows over every step (rows are independent)."""
+import ast
+import functools
+import os
+
+import numpy as np
+import pytest
+
+from workloads import synth
+
+from gpu_util import GpuGate, compare
+
+pytestmark = pytest.mark.gpu
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+sys_path_golden = os.path.join(GOLDEN)
+
+
+def _plans():
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(GOLDEN, "make_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    return mod.PLANS
+
+
+PLANS = _plans()
+
+
+@functools.lru_cache(maxsize=2)
+def _head(seed, which, V, H):
+    return synth.lm_head(seed, which, V, H)
+
+
+@pytest.mark.parametrize("name", sorted(PLANS))
+def test_full_size_against_stored_oracle(name):
+    cfg, over, T_head, rows, T = PLANS[name]
+    cfg = cfg.with_(**over)
+    z = np.load(os.path.join(GOLDEN, f"oracle_{name}.npz"))
+    meta = ast.literal_eval(str(z["meta"]))
+    assert meta["B"] == cfg.B and meta["T"] == T and meta["V"] == cfg.V and meta["w"] == cfg.w
+    assert meta["d_min"] == cfg.d_min and meta["seed"] == cfg.seed
+    assert meta["tau"] == float(np.float32(cfg.tau)), "stored oracle run used another threshold"
+
+    wl = synth.Workload(cfg, T=T, heads=False)
+    Ws, Wl = _head(cfg.seed, 0, cfg.V, cfg.H_small), _head(cfg.seed, 1, cfg.V, cfg.H_large)
+    with GpuGate(cfg, Ws, Wl) as g:
+        info = g.E.ead_launch_info(g.ctx)
+        out = g.run(wl.h_small, wl.h_large, "run")
+    assert info["ctas"] >= 100
+
+    ora_rows = {k[5:]: z[k] for k in z.files if k.startswith("rows_")}
+    log = compare(out, ora_rows, cfg.tau)
+    cells = log["cells"]
+    if T_head:
+        ora_head = {k[5:]: z[k] for k in z.files if k.startswith("head_")}
+        log_h = compare({k: v[:T_head] for k, v in out.items()}, ora_head, cfg.tau)
+        cells += log_h["cells"]
+        for k in ("token_near_ties", "switch_near_ties"):
+            log[k] += log_h[k]
+        log["max_H_err"] = max(log["max_H_err"], log_h["max_H_err"])
+    print(f"{name}: {cells} cells compared, max |dH| {log['max_H_err']:.2e}, "
+          f"token near-ties {log['token_near_ties']}, switch near-ties {log['switch_near_ties']}, "
+          f"large-head share {out['used'].mean():.3f}")
+    assert cells >= 0.9 * (T_head * cfg.B + len(rows) * T)
+    assert len(log["token_near_ties"]) + len(log["switch_near_ties"]) <= 3
