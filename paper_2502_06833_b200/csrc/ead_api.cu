@@ -71,6 +71,7 @@ struct ead_ctx {
     cudaStream_t cap_stream = nullptr;     // capture happens on a private stream
     int G = 0, a_rows = 0, stages = 0, slots_stride = 0;
     int small_cols = 0;                    // > 0: swapped-operand kernel with this many batch columns
+    int small_slots = 0;                   // partial slots per row it writes (one per CTA and epilogue warp)
     size_t smem_bytes = 0;
     const void *W[2] = {nullptr, nullptr};
     // device state and scratch (owned)
@@ -80,7 +81,7 @@ struct ead_ctx {
     int32_t *c = nullptr, *nfill = nullptr, *perm = nullptr, *part_i = nullptr;
     float *ring = nullptr, *part_m = nullptr, *part_s = nullptr, *part_t = nullptr;
     uint16_t *hc[2] = {nullptr, nullptr};
-    CUtensorMap tmA[2], tmW[2], tmT[2];
+    CUtensorMap tmA[2], tmW[2], tmT[2], tmP[2];   // hidden rows; W boxes of 256|128, 16 and 32 rows
     cudaGraphExec_t g_one = nullptr, g_chunk = nullptr;
     int64_t launches = 0;
     // staging of ead_run_host (allocated on first use)
@@ -129,18 +130,21 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     lp.part_s = x->part_s;
     lp.part_t = x->part_t;
     lp.part_i = x->part_i;
-#define EAD_LAUNCH_LMHEAD(kernel)                                                                              \
-    kernel<<<x->G, kLmheadThreads, x->smem_bytes, s>>>(x->tmA[0], x->tmA[1], x->tmW[0], x->tmW[1], x->tmT[0], \
-                                                       x->tmT[1], lp)
+#define EAD_LAUNCH_SMALL(NB)                                                                                  \
+    ead_lmhead_small_kernel<NB><<<x->G, kLmheadThreads, x->smem_bytes, s>>>(                                    \
+        x->tmA[0], x->tmA[1], x->tmW[0], x->tmW[1], x->tmP[0], x->tmP[1], lp)
     switch (x->small_cols) {
-        case 0: EAD_LAUNCH_LMHEAD(ead_lmhead_kernel); break;
-        case 1: EAD_LAUNCH_LMHEAD(ead_lmhead_small_kernel<1>); break;
-        case 2: EAD_LAUNCH_LMHEAD(ead_lmhead_small_kernel<2>); break;
-        case 4: EAD_LAUNCH_LMHEAD(ead_lmhead_small_kernel<4>); break;
-        case 8: EAD_LAUNCH_LMHEAD(ead_lmhead_small_kernel<8>); break;
-        default: EAD_LAUNCH_LMHEAD(ead_lmhead_small_kernel<16>); break;
+        case 0:
+            ead_lmhead_kernel<<<x->G, kLmheadThreads, x->smem_bytes, s>>>(x->tmA[0], x->tmA[1], x->tmW[0], x->tmW[1],
+                                                                          x->tmT[0], x->tmT[1], lp);
+            break;
+        case 1: EAD_LAUNCH_SMALL(1); break;
+        case 2: EAD_LAUNCH_SMALL(2); break;
+        case 4: EAD_LAUNCH_SMALL(4); break;
+        case 8: EAD_LAUNCH_SMALL(8); break;
+        default: EAD_LAUNCH_SMALL(16); break;
     }
-#undef EAD_LAUNCH_LMHEAD
+#undef EAD_LAUNCH_SMALL
     if (ev) cudaEventRecord(ev[2], s);
 
     GateParams gp{};
@@ -151,6 +155,7 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     gp.unit = c.unit;
     gp.G = x->G;
     gp.slots_stride = x->slots_stride;
+    gp.n_slots = x->small_slots;
     gp.tau = c.tau;
     gp.ctl = x->ctl;
     gp.args = x->args;
@@ -164,7 +169,10 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     gp.nfill = x->nfill;
     gp.ring = x->ring;
     const int rows_per_block = kGateThreads / 32;
-    ead_merge_gate_kernel<<<(c.B + rows_per_block - 1) / rows_per_block, kGateThreads, 0, s>>>(gp);
+    if (x->small_cols)
+        ead_merge_gate_wide_kernel<<<c.B, kGateThreads, 0, s>>>(gp);
+    else
+        ead_merge_gate_kernel<<<(c.B + rows_per_block - 1) / rows_per_block, kGateThreads, 0, s>>>(gp);
     if (ev) cudaEventRecord(ev[3], s);
     return cudaGetLastError() == cudaSuccess ? EAD_OK : EAD_ECUDA;
 }
@@ -328,7 +336,7 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     x->stream = static_cast<cudaStream_t>(cfg->stream);
     x->W[0] = W_small;
     x->W[1] = W_large;
-    x->G = prop.multiProcessorCount;
+    x->G = std::min(prop.multiProcessorCount, kMaxCtas);
     if ((cfg->B + kTileM - 1) / kTileM > x->G) {   // the work split needs one CTA per row block at least
         delete x;
         return EAD_EINVALID_ARG;
@@ -340,13 +348,15 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
         // latency regime: swapped-operand kernel, batch columns rounded up to a power of two
         x->small_cols = 1;
         while (x->small_cols < cfg->B) x->small_cols *= 2;
-        x->a_rows = kSmallN;
-        stage_bytes = kSmallStageBytes;
+        x->a_rows = cfg->B <= 8 ? 8 : kSmallN;
+        stage_bytes = small_stage_bytes(x->a_rows);
+        x->small_slots = x->G * kSmallSlotsPerCta;
+        x->slots_stride = (x->small_slots + 31) & ~31;
     } else {
         x->a_rows = std::min(kTileM, (cfg->B + 7) & ~7);
         stage_bytes = static_cast<size_t>(x->a_rows) * kBlockK * 2 + kWTileBytes;
     }
-    x->stages = static_cast<int>(std::min<size_t>(kMaxStages, (smem_max - kSmemCtrlBytes - 1024) / stage_bytes));
+    x->stages = static_cast<int>(std::min<size_t>(kMaxStages, (smem_max - kSmemCtrlBytes - 1024 - 1024) / stage_bytes));
     x->smem_bytes = kSmemCtrlBytes + 1024 + x->stages * stage_bytes;
 
     const int B = cfg->B;
@@ -386,7 +396,8 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     for (int m = 0; m < 2; ++m) {
         if (!encode_bf16_2d(&x->tmA[m], x->hc[m], Bpad, Hm[m], x->a_rows) ||
             !encode_bf16_2d(&x->tmW[m], x->W[m], cfg->V, Hm[m], wbox) ||
-            !encode_bf16_2d(&x->tmT[m], x->W[m], cfg->V, Hm[m], kUnit))
+            !encode_bf16_2d(&x->tmT[m], x->W[m], cfg->V, Hm[m], kUnit) ||
+            !encode_bf16_2d(&x->tmP[m], x->W[m], cfg->V, Hm[m], kSmallSegRows))
             return fail(EAD_ECUDA);
     }
     // the attribute belongs to the kernel on this device, not to the context: ask for the

@@ -11,6 +11,7 @@ constexpr int kTileM = 128;        // batch rows per accumulator tile (MMA M = T
 constexpr int kBlockK = 64;        // hidden elements per pipeline stage (128 B of bf16)
 constexpr int kUnit = 16;          // granularity of a CTA's vocabulary range (MMA N step)
 constexpr int kMaxStages = 8;
+constexpr int kMaxCtas = 256;         // upper bound on the LM-head grid (one CTA per SM)
 constexpr int kWTileBytes = kTileN * kBlockK * 2;   // 32 KiB
 constexpr int kSmemCtrlBytes = 1024;
 constexpr int kLmheadThreads = 192;                 // TMA warp, MMA warp, 4 epilogue warps
@@ -105,7 +106,7 @@ struct LmheadParams {
     int32_t a_rows;        // rows of the hidden-state TMA box (multiple of 8, <= 128)
     int32_t n_cols;        // small-batch kernel: batch columns kept per thread (power of two <= 16)
     int32_t stages;
-    int32_t slots_stride;  // partial slots per row (>= CTAs)
+    int32_t slots_stride;  // partial slots per row (>= CTAs x slots per CTA)
     int32_t B;
     const StepCtl *ctl;
     StepCtl *ctl_rw;

@@ -98,6 +98,7 @@ ead_compact_kernel(StepCtl *ctl, const RunArgs *args, const uint8_t *flag, int B
 
 struct GateParams {
     int32_t B, V, w, d_min, unit, G, slots_stride;
+    int32_t n_slots;           // > 0: partial slots per row as written by the small-batch kernel
     float tau;
     StepCtl *ctl;
     const RunArgs *args;
@@ -110,44 +111,11 @@ struct GateParams {
     float *ring;
 };
 
-// One warp per compacted row.
-__global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const GateParams p)
+// Everything after the merge for one compacted row (executed by one thread): Eq. 2 in the
+// fused form, then the tail of Algorithm 1's loop body (window, counter, Eq. 4), state update
+// and outputs scattered back to the caller's row.
+__device__ __forceinline__ void finish_row(const GateParams &p, int m, int r, const Partial &acc, int t_step)
 {
-    const int lane = threadIdx.x & 31;
-    const int i = blockIdx.x * (kGateThreads / 32) + (threadIdx.x >> 5);
-    const int n0 = p.ctl->n[0], n1 = p.ctl->n[1];
-    const int t_step = p.ctl->cur_t;
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        if (n0 + n1 != p.B) atomicOr(&p.ctl->status, kStatusBadCount);
-        p.ctl->step = t_step + 1;                 // nobody in this kernel reads `step`
-    }
-    if (i >= p.B || n0 + n1 != p.B) return;
-    const int m = i < n0 ? 0 : 1;
-    const int r = m ? i - n0 : i;
-    const int n_m = m ? n1 : n0;
-    const int R = (n_m + kTileM - 1) / kTileM;
-    int g = p.G / R;
-    if (g < 1) g = 1;
-
-    // ---- cross-CTA merge, fixed order: each lane folds its slots in ascending
-    //      order, then a butterfly over the lanes (no float atomics: deterministic)
-    const size_t base = (static_cast<size_t>(m) * p.B + r) * p.slots_stride;
-    Partial acc{kNegSentinel, 0.f, 0.f, 0x7fffffff};
-    for (int s = lane; s < g; s += 32) {
-        const Partial q{p.part_m[base + s], p.part_s[base + s], p.part_t[base + s], p.part_i[base + s]};
-        acc = merge_partial(acc, q);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        Partial q;
-        q.m = __shfl_xor_sync(0xffffffffu, acc.m, o);
-        q.s = __shfl_xor_sync(0xffffffffu, acc.s, o);
-        q.t = __shfl_xor_sync(0xffffffffu, acc.t, o);
-        q.idx = __shfl_xor_sync(0xffffffffu, acc.idx, o);
-        acc = merge_partial(acc, q);
-    }
-    if (lane != 0) return;
-
     // ---- Eq. 2 in the fused form  H = ln Z - E_p[z] = ln s - t / (s log2 e)   (nats)
     float H = logf(acc.s) - acc.t / (acc.s * kLog2e);
     const bool finite = isfinite(H) && acc.s > 0.f;
@@ -191,6 +159,84 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const Gate
     if (p.args->Hbar) p.args->Hbar[o] = Hbar;
     if (p.args->used) p.args->used[o] = static_cast<uint8_t>(used);
     if (p.args->next) p.args->next[o] = static_cast<uint8_t>(model);
+}
+
+__device__ __forceinline__ Partial warp_merge(Partial acc)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Partial q;
+        q.m = __shfl_xor_sync(0xffffffffu, acc.m, o);
+        q.s = __shfl_xor_sync(0xffffffffu, acc.s, o);
+        q.t = __shfl_xor_sync(0xffffffffu, acc.t, o);
+        q.idx = __shfl_xor_sync(0xffffffffu, acc.idx, o);
+        acc = merge_partial(acc, q);
+    }
+    return acc;
+}
+
+// One warp per compacted row: partials of ead_lmhead_kernel (one slot per CTA of the row's group).
+__global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const GateParams p)
+{
+    const int lane = threadIdx.x & 31;
+    const int i = blockIdx.x * (kGateThreads / 32) + (threadIdx.x >> 5);
+    const int n0 = p.ctl->n[0], n1 = p.ctl->n[1];
+    const int t_step = p.ctl->cur_t;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        if (n0 + n1 != p.B) atomicOr(&p.ctl->status, kStatusBadCount);
+        p.ctl->step = t_step + 1;                 // nobody in this kernel reads `step`
+    }
+    if (i >= p.B || n0 + n1 != p.B) return;
+    const int m = i < n0 ? 0 : 1;
+    const int r = m ? i - n0 : i;
+    const int n_m = m ? n1 : n0;
+    const int R = (n_m + kTileM - 1) / kTileM;
+    int g = p.G / R;
+    if (g < 1) g = 1;
+
+    // ---- cross-CTA merge, fixed order: each lane folds its slots in ascending
+    //      order, then a butterfly over the lanes (no float atomics: deterministic)
+    const size_t base = (static_cast<size_t>(m) * p.B + r) * p.slots_stride;
+    Partial acc{kNegSentinel, 0.f, 0.f, 0x7fffffff};
+    for (int s = lane; s < g; s += 32) {
+        const Partial q{p.part_m[base + s], p.part_s[base + s], p.part_t[base + s], p.part_i[base + s]};
+        acc = merge_partial(acc, q);
+    }
+    acc = warp_merge(acc);
+    if (lane == 0) finish_row(p, m, r, acc, t_step);
+}
+
+// One block per compacted row: the 4 G partials of the small-batch kernel.  Thread t folds slots t, t + 256, ... in ascending order, then lanes, then warps:
+// a fixed order again.
+__global__ void __launch_bounds__(kGateThreads) ead_merge_gate_wide_kernel(const GateParams p)
+{
+    __shared__ Partial wsum[kGateThreads / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int i = blockIdx.x;
+    const int n0 = p.ctl->n[0], n1 = p.ctl->n[1];
+    const int t_step = p.ctl->cur_t;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        if (n0 + n1 != p.B) atomicOr(&p.ctl->status, kStatusBadCount);
+        p.ctl->step = t_step + 1;
+    }
+    if (i >= p.B || n0 + n1 != p.B) return;
+    const int m = i < n0 ? 0 : 1;
+    const int r = m ? i - n0 : i;
+    const size_t base = (static_cast<size_t>(m) * p.B + r) * p.slots_stride;
+    Partial acc{kNegSentinel, 0.f, 0.f, 0x7fffffff};
+    for (int s = threadIdx.x; s < p.n_slots; s += kGateThreads) {
+        const Partial q{p.part_m[base + s], p.part_s[base + s], p.part_t[base + s], p.part_i[base + s]};
+        acc = merge_partial(acc, q);
+    }
+    acc = warp_merge(acc);
+    if (lane == 0) wsum[warp] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        acc = wsum[0];
+#pragma unroll
+        for (int k = 1; k < kGateThreads / 32; ++k) acc = merge_partial(acc, wsum[k]);
+        finish_row(p, m, r, acc, t_step);
+    }
 }
 
 }  // namespace ead

@@ -33,6 +33,7 @@ struct SmemCtrl {
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint64_t drain;
+    int32_t tile[2][4];         // small-batch kernel: {first row, end row, range} of this CTA
     uint32_t tmem_base;
     uint32_t abort;
 };

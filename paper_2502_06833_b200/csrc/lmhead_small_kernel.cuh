@@ -5,32 +5,44 @@
 // This kernel swaps the operands instead: MMA M (TMEM lanes) = 128 vocabulary rows of W,
 // MMA N (TMEM columns) = 16 batch columns, K = hidden, so the tensor work is 16x smaller
 // and W is the only operand of any size.  One epilogue thread owns one vocabulary row of
-// every tile (rows r, r + 128, ... of the CTA's range) and keeps NB running statistics,
-// one per sequence; they are merged across the 128 threads once, at the end of the range.
-// The result is written in the same per-CTA partial format as ead_lmhead_kernel, so the
-// merge + gate kernel does not care which of the two produced it.
+// a tile and NB statistics, one per sequence.
 //
-// Pipeline: per K block of 128 hidden elements one stage = two 64-wide W boxes (128 rows
-// each, 16 KiB) + two 64-wide boxes of the compacted hidden rows (16 rows, 2 KiB); TMEM
-// holds two 16-column accumulators so that the epilogue overlaps the next tile's MMAs.
+// The statistics run across all tiles of the CTA's range; at the end of a head every epilogue
+// warp reduces its 32 threads and writes one partial per sequence (slot = 4 * CTA + warp),
+// in the format of ead_lmhead_kernel, so the merge + gate kernel does not care which of the
+// two kernels produced it.
+//
+// Work distribution: the vocabulary is cut into G contiguous ranges of (almost) equal length,
+// in units of 32 rows.  (SMs do not all get the same share of HBM bandwidth - finish times of
+// an equal split spread by +-10 % - but which SMs lag changes with the split itself, so
+// ranges sized from a measurement do not converge, and the lagging SMs speed up once the
+// others are done, so the HBM stays busy; measured cost of the imbalance against dynamic
+// scheduling of 256 KB units: 3-4 %.)
+//
+// Pipeline: per K block of 128 hidden elements one stage = two 64-wide W boxes (<= 128 rows
+// each, 16 KiB) + two 64-wide boxes of the compacted hidden rows (8 rows if B <= 8, else 16;
+// the MMA's N = 16 then reads the following kilobyte as rows 8-15, which only feeds
+// accumulator columns nobody reads).  TMEM holds two 16-column accumulators so that the
+// epilogue overlaps the next tile's MMAs.
 #pragma once
 #include "lmhead_kernel.cuh"
 
 namespace ead {
 
 constexpr int kSmallTileRows = 128;                    // vocabulary rows per tile (MMA M)
+constexpr int kSmallSegRows = 32;                      // granularity of a CTA's vocabulary range
+constexpr int kSmallSlotsPerCta = 4;                   // one partial per epilogue warp
 constexpr int kSmallN = 16;                            // batch columns (MMA N)
 constexpr int kSmallBlockK = 128;                      // hidden elements per stage
-constexpr int kSmallHBytes = kSmallN * 64 * 2;         // one 64-wide box of hidden rows: 2 KiB
 constexpr int kSmallWBytes = kSmallTileRows * 64 * 2;  // one 64-wide box of W rows: 16 KiB
-constexpr int kSmallStageBytes = 2 * kSmallHBytes + 2 * kSmallWBytes;   // 36 KiB
 constexpr int kSmallTmemCols = 32;                     // 2 accumulators x 16 columns
+__host__ __device__ constexpr int small_stage_bytes(int h_rows) { return 2 * h_rows * 128 + 2 * kSmallWBytes; }
 
 template <int NB>
 __global__ void __launch_bounds__(kLmheadThreads, 1)
 ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
                         const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
-                        const __grid_constant__ CUtensorMap tmT0, const __grid_constant__ CUtensorMap tmT1,
+                        const __grid_constant__ CUtensorMap tmP0, const __grid_constant__ CUtensorMap tmP1,
                         const LmheadParams p)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -38,13 +50,14 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                                                 ~static_cast<uintptr_t>(1023));
     SmemCtrl *ctrl = reinterpret_cast<SmemCtrl *>(smem);
     uint8_t *stage0 = smem + kSmemCtrlBytes;
-    __shared__ Partial xwarp[4][NB];
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int cta = blockIdx.x;
     const int G = gridDim.x;
     const int stages = p.stages;
+    const uint32_t h_slab = static_cast<uint32_t>(p.a_rows) * 128;      // hidden rows of one 64-wide K slab
+    const uint32_t stage_bytes = 2 * h_slab + 2 * kSmallWBytes;
+    StepCtl *ctl = p.ctl_rw;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < stages; ++i) {
@@ -62,7 +75,7 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
     if (warp == 0 && lane == 0) {
         tma_prefetch_desc(&tmA0); tma_prefetch_desc(&tmA1);
         tma_prefetch_desc(&tmW0); tma_prefetch_desc(&tmW1);
-        tma_prefetch_desc(&tmT0); tma_prefetch_desc(&tmT1);
+        tma_prefetch_desc(&tmP0); tma_prefetch_desc(&tmP1);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&ctrl->tmem_base), kSmallTmemCols);
@@ -72,9 +85,12 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&ctrl->tmem_base);
-
+    const int v_pad = (p.V + kSmallSegRows - 1) / kSmallSegRows * kSmallSegRows;
+    const int n_seg = v_pad / kSmallSegRows;
+    const int cta = blockIdx.x;
+    const int row_begin = static_cast<int>(static_cast<long long>(n_seg) * cta / G) * kSmallSegRows;
+    const int row_end = static_cast<int>(static_cast<long long>(n_seg) * (cta + 1) / G) * kSmallSegRows;
     const int n_rows[2] = {p.ctl->n[0], p.ctl->n[1]};
-    StepCtl *ctl = p.ctl_rw;
 
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer
@@ -83,37 +99,37 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
             uint32_t it = 0;
             bool ok = true;
             for (int m = 0; m < 2 && ok; ++m) {
-                const HeadSplit sp = split_head(cta, G, n_rows[m], p.V);   // n <= 16: one row block
-                if (!sp.active) continue;
+                if (n_rows[m] <= 0) continue;
                 const CUtensorMap *tA = m ? &tmA1 : &tmA0;
                 const CUtensorMap *tW = m ? &tmW1 : &tmW0;
-                const CUtensorMap *tT = m ? &tmT1 : &tmT0;
+                const CUtensorMap *tP = m ? &tmP1 : &tmP0;
                 const int kblocks = (p.H[m] + kSmallBlockK - 1) / kSmallBlockK;
-                for (int row0 = sp.col_begin; row0 < sp.col_end && ok; row0 += kSmallTileRows) {
-                    const int nrows = min(kSmallTileRows, sp.col_end - row0);
-                    const uint32_t tx = 2 * kSmallHBytes + 2 * static_cast<uint32_t>(nrows) * 128;
+                for (int row0 = row_begin; row0 < row_end && ok; row0 += kSmallTileRows) {
+                    const int nrows = min(kSmallTileRows, row_end - row0);        // multiple of 32
+                    const uint32_t tx = 2 * (h_slab + static_cast<uint32_t>(nrows) * 128);
                     for (int kb = 0; kb < kblocks; ++kb, ++it) {
                         const uint32_t s = it % stages;
                         const uint32_t ph = (it / stages) & 1u;
                         if (!wait_bar(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, ctl)) { ok = false; break; }
                         const uint32_t bar = smem_u32(&ctrl->full[s]);
-                        const uint32_t sa = smem_u32(stage0 + static_cast<size_t>(s) * kSmallStageBytes);
+                        const uint32_t sa = smem_u32(stage0 + static_cast<size_t>(s) * stage_bytes);
                         mbar_arrive_expect_tx(bar, tx);
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
                             const int k0 = kb * kSmallBlockK + h * 64;
-                            tma_load_2d(sa + h * kSmallHBytes, tA, k0, 0, bar, pol_keep);
-                            const uint32_t wdst = sa + 2 * kSmallHBytes + h * kSmallWBytes;
+                            tma_load_2d(sa + h * h_slab, tA, k0, 0, bar, pol_keep);
+                            const uint32_t wdst = sa + 2 * h_slab + h * kSmallWBytes;
                             if (nrows == kSmallTileRows) {
                                 tma_load_2d(wdst, tW, k0, row0, bar, pol_keep);
                             } else {
-                                for (int j = 0; j < nrows; j += kUnit)
-                                    tma_load_2d(wdst + j * 128, tT, k0, row0 + j, bar, pol_keep);
+                                for (int j = 0; j < nrows; j += kSmallSegRows)
+                                    tma_load_2d(wdst + j * 128, tP, k0, row0 + j, bar, pol_keep);
                             }
                         }
                     }
                 }
             }
+            // Before the CTA retires, every copy issued above must have landed.
             const uint32_t pending = it < static_cast<uint32_t>(stages) ? it : stages;
             for (uint32_t k = 0; k < pending; ++k) {
                 const uint32_t j = it - 1 - k;
@@ -127,10 +143,9 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
             bool ok = true;
             const uint32_t idesc = umma_idesc_bf16_m128(kSmallN);
             for (int m = 0; m < 2 && ok; ++m) {
-                const HeadSplit sp = split_head(cta, G, n_rows[m], p.V);
-                if (!sp.active) continue;
+                if (n_rows[m] <= 0) continue;
                 const int kblocks = (p.H[m] + kSmallBlockK - 1) / kSmallBlockK;
-                for (int row0 = sp.col_begin; row0 < sp.col_end && ok; row0 += kSmallTileRows, ++tc) {
+                for (int row0 = row_begin; row0 < row_end && ok; row0 += kSmallTileRows, ++tc) {
                     const uint32_t buf = tc & 1u;
                     if (!wait_bar(smem_u32(&ctrl->tmem_empty[buf]), ((tc >> 1) & 1u) ^ 1u, ctrl, ctl)) {
                         ok = false;
@@ -145,11 +160,11 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                             break;
                         }
                         tc_fence_after_sync();
-                        const uint32_t sa = smem_u32(stage0 + static_cast<size_t>(s) * kSmallStageBytes);
+                        const uint32_t sa = smem_u32(stage0 + static_cast<size_t>(s) * stage_bytes);
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            const uint64_t dh = umma_smem_desc(sa + h * kSmallHBytes);                      // B: hidden rows
-                            const uint64_t dw = umma_smem_desc(sa + 2 * kSmallHBytes + h * kSmallWBytes);   // A: W rows
+                            const uint64_t dh = umma_smem_desc(sa + h * h_slab);                         // B: hidden rows
+                            const uint64_t dw = umma_smem_desc(sa + 2 * h_slab + h * kSmallWBytes);      // A: W rows
 #pragma unroll
                             for (int k = 0; k < 4; ++k)
                                 umma_bf16(d_tmem, dw + 2 * k, dh + 2 * k, idesc, (kb | h | k) != 0);
@@ -159,20 +174,17 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                     if (ok) umma_commit(smem_u32(&ctrl->tmem_full[buf]));
                 }
             }
+            // All MMAs must have finished before TMEM is released.
             umma_commit(smem_u32(&ctrl->drain));
             wait_bar(smem_u32(&ctrl->drain), 0u, ctrl, ctl);
         }
     } else {
         // ------------------------------------------------------------- epilogue
-        const int quad = warp & 3;
-        const int ew = warp - 2;                       // 0..3
+        const int quad = warp & 3;                     // TMEM lane quadrant this warp may read
         uint32_t tc = 0;
         bool ok = true;
-        // Every epilogue warp passes the same named barriers whatever happened to its waits,
-        // so a warp that gave up cannot leave the others stuck at one.
-        for (int m = 0; m < 2; ++m) {
-            const HeadSplit sp = split_head(cta, G, n_rows[m], p.V);
-            if (!sp.active) continue;
+        for (int m = 0; m < 2 && ok; ++m) {
+            if (n_rows[m] <= 0) continue;
             float sm[NB], ss[NB], stt[NB];
             int sidx[NB];
 #pragma unroll
@@ -182,8 +194,8 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                 stt[j] = 0.f;
                 sidx[j] = 0x7fffffff;
             }
-            const int row_limit = min(p.V, sp.col_end);
-            for (int row0 = sp.col_begin; row0 < sp.col_end && ok; row0 += kSmallTileRows, ++tc) {
+            for (int row0 = row_begin; row0 < row_end && ok; row0 += kSmallTileRows, ++tc) {
+                const int nrows = min(kSmallTileRows, row_end - row0);
                 const uint32_t buf = tc & 1u;
                 if (!wait_bar_warp(smem_u32(&ctrl->tmem_full[buf]), (tc >> 1) & 1u, ctrl, ctl, lane)) {
                     ok = false;
@@ -195,8 +207,9 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[buf]));
-                const int row = row0 + quad * 32 + lane;          // vocabulary entry of this thread
-                if (row < row_limit) {
+                const int r_in = quad * 32 + lane;
+                const int row = row0 + r_in;                       // vocabulary entry of this thread
+                if (r_in < nrows && row < p.V) {
 #pragma unroll
                     for (int j = 0; j < NB; ++j) {
                         const float z = v[j];
@@ -213,7 +226,8 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                 }
                 __syncwarp();
             }
-            // ---- merge the 128 per-thread statistics of every sequence: lanes, then warps
+            if (!ok) break;
+            // ---- end of the head: reduce the 32 threads of this warp, one partial per sequence
 #pragma unroll
             for (int j = 0; j < NB; ++j) {
                 Partial acc{sm[j], ss[j], stt[j], sidx[j]};
@@ -226,19 +240,15 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                     q.idx = __shfl_xor_sync(0xffffffffu, acc.idx, o);
                     acc = merge_partial(acc, q);
                 }
-                if (lane == 0) xwarp[ew][j] = acc;
+                if (lane == 0 && j < n_rows[m]) {
+                    const size_t o = (static_cast<size_t>(m) * p.B + j) * p.slots_stride +
+                                     cta * kSmallSlotsPerCta + quad;
+                    p.part_m[o] = acc.m;
+                    p.part_s[o] = acc.s;
+                    p.part_t[o] = acc.t;
+                    p.part_i[o] = acc.idx;
+                }
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");        // the four epilogue warps only
-            if (ew == 0 && lane < NB && lane < n_rows[m] && ok) {
-                Partial acc = xwarp[0][lane];
-                for (int k = 1; k < 4; ++k) acc = merge_partial(acc, xwarp[k][lane]);
-                const size_t o = (static_cast<size_t>(m) * p.B + lane) * p.slots_stride + sp.slot;
-                p.part_m[o] = acc.m;
-                p.part_s[o] = acc.s;
-                p.part_t[o] = acc.t;
-                p.part_i[o] = acc.idx;
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");        // xwarp is reused by the next head
         }
     }
 
