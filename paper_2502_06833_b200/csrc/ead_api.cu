@@ -104,15 +104,39 @@ namespace {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Launches `kernel`; with `pdl` the launch carries the programmatic-stream-serialization
+// attribute: the kernel may start while its predecessor in the stream is still running and
+// synchronises with it through griddepcontrol.wait.
+template <typename... KArgs, typename... Args>
+cudaError_t launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool pdl,
+                   Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // The three kernels of one gate step, in stream order.  With `ev` (4 events) the
-// boundaries between the kernels are recorded for timing.
+// boundaries between the kernels are recorded for timing and the kernels do not overlap;
+// otherwise each kernel's set-up overlaps the tail of the one before it.
 int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
 {
     const ead_config &c = x->cfg;
+    const bool pdl = ev == nullptr;
     const int cgrid = std::min(c.B, 4 * x->G);
+    cudaError_t e = cudaSuccess;
     if (ev) cudaEventRecord(ev[0], s);
-    ead_compact_kernel<<<cgrid, kCompactThreads, static_cast<size_t>(c.B) * sizeof(int32_t), s>>>(
-        x->ctl, x->args, x->flag, c.B, c.H_small, c.H_large, x->hc[0], x->hc[1], x->perm);
+    e = launch(ead_compact_kernel, dim3(cgrid), dim3(kCompactThreads), static_cast<size_t>(c.B) * sizeof(int32_t), s, pdl,
+               x->ctl, x->args, x->flag, c.B, c.H_small, c.H_large, x->hc[0], x->hc[1], x->perm);
+    if (e != cudaSuccess) return EAD_ECUDA;
     if (ev) cudaEventRecord(ev[1], s);
 
     LmheadParams lp{};
@@ -130,13 +154,14 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     lp.part_s = x->part_s;
     lp.part_t = x->part_t;
     lp.part_i = x->part_i;
+    const dim3 lgrid(x->G), lblock(kLmheadThreads);
 #define EAD_LAUNCH_SMALL(NB)                                                                                  \
-    ead_lmhead_small_kernel<NB><<<x->G, kLmheadThreads, x->smem_bytes, s>>>(                                    \
-        x->tmA[0], x->tmA[1], x->tmW[0], x->tmW[1], x->tmP[0], x->tmP[1], lp)
+    e = launch(ead_lmhead_small_kernel<NB>, lgrid, lblock, x->smem_bytes, s, pdl, x->tmA[0], x->tmA[1], x->tmW[0], \
+               x->tmW[1], x->tmP[0], x->tmP[1], lp)
     switch (x->small_cols) {
         case 0:
-            ead_lmhead_kernel<<<x->G, kLmheadThreads, x->smem_bytes, s>>>(x->tmA[0], x->tmA[1], x->tmW[0], x->tmW[1],
-                                                                          x->tmT[0], x->tmT[1], lp);
+            e = launch(ead_lmhead_kernel, lgrid, lblock, x->smem_bytes, s, pdl, x->tmA[0], x->tmA[1], x->tmW[0],
+                       x->tmW[1], x->tmT[0], x->tmT[1], lp);
             break;
         case 1: EAD_LAUNCH_SMALL(1); break;
         case 2: EAD_LAUNCH_SMALL(2); break;
@@ -145,6 +170,7 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
         default: EAD_LAUNCH_SMALL(16); break;
     }
 #undef EAD_LAUNCH_SMALL
+    if (e != cudaSuccess) return EAD_ECUDA;
     if (ev) cudaEventRecord(ev[2], s);
 
     GateParams gp{};
@@ -170,9 +196,11 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     gp.ring = x->ring;
     const int rows_per_block = kGateThreads / 32;
     if (x->small_cols)
-        ead_merge_gate_wide_kernel<<<c.B, kGateThreads, 0, s>>>(gp);
+        e = launch(ead_merge_gate_wide_kernel, dim3(c.B), dim3(kGateThreads), 0, s, pdl, gp);
     else
-        ead_merge_gate_kernel<<<(c.B + rows_per_block - 1) / rows_per_block, kGateThreads, 0, s>>>(gp);
+        e = launch(ead_merge_gate_kernel, dim3((c.B + rows_per_block - 1) / rows_per_block), dim3(kGateThreads), 0, s,
+                   pdl, gp);
+    if (e != cudaSuccess) return EAD_ECUDA;
     if (ev) cudaEventRecord(ev[3], s);
     return cudaGetLastError() == cudaSuccess ? EAD_OK : EAD_ECUDA;
 }

@@ -7,6 +7,7 @@
 //   ead_set_args_kernel, ead_reset_kernel   bookkeeping
 #pragma once
 #include "ead_internal.cuh"
+#include "ptx_sm100.cuh"
 
 namespace ead {
 
@@ -49,6 +50,8 @@ ead_compact_kernel(StepCtl *ctl, const RunArgs *args, const uint8_t *flag, int B
     extern __shared__ int32_t pos_sh[];          // [B]: position | model << 30
     __shared__ int32_t warp_tot[kCompactThreads / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    griddep_launch_dependents();                 // the LM-head kernel may set itself up meanwhile
+    griddep_wait();                              // flags and step counter come from the previous step
     const int step = ctl->step;
     const int idx = step - args->run_base;
 
@@ -180,6 +183,8 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const Gate
 {
     const int lane = threadIdx.x & 31;
     const int i = blockIdx.x * (kGateThreads / 32) + (threadIdx.x >> 5);
+    griddep_launch_dependents();
+    griddep_wait();                              // partials of the LM-head kernel
     const int n0 = p.ctl->n[0], n1 = p.ctl->n[1];
     const int t_step = p.ctl->cur_t;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -213,6 +218,8 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_wide_kernel(const
     __shared__ Partial wsum[kGateThreads / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int i = blockIdx.x;
+    griddep_launch_dependents();
+    griddep_wait();                              // partials of the LM-head kernel
     const int n0 = p.ctl->n[0], n1 = p.ctl->n[1];
     const int t_step = p.ctl->cur_t;
     if (blockIdx.x == 0 && threadIdx.x == 0) {

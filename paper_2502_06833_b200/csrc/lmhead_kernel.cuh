@@ -173,6 +173,9 @@ ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
     tc_fence_after_sync();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&ctrl->tmem_base);
 
+    // Everything above touched no global memory: it may overlap the kernels before this one.
+    griddep_wait();
+    griddep_launch_dependents();
     const int n_rows[2] = {p.ctl->n[0], p.ctl->n[1]};
     StepCtl *ctl = p.ctl_rw;
 

@@ -85,6 +85,9 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&ctrl->tmem_base);
+    // Everything above touched no global memory: it may overlap the kernels before this one.
+    griddep_wait();
+    griddep_launch_dependents();
     const int v_pad = (p.V + kSmallSegRows - 1) / kSmallSegRows * kSmallSegRows;
     const int n_seg = v_pad / kSmallSegRows;
     const int cta = blockIdx.x;

@@ -20,6 +20,19 @@ __device__ __forceinline__ uint64_t globaltimer_ns()
     return t;
 }
 
+// ----------------------------------------------------------------- programmatic dependent launch
+// No-ops unless the kernel was launched with the programmatic-stream-serialization attribute.
+// wait: blocks until the grids this one depends on have completed and their writes are visible.
+// launch_dependents: lets the next kernel in the stream start (up to its own wait) early.
+__device__ __forceinline__ void griddep_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void griddep_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ----------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
