@@ -38,7 +38,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per LM-head launch from the committed ncu
 # capture of the same kernel (profiles/), keyed by config; None until captured for the
 # kernel as it stands.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama_b1": 1.05484e9}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
 
 
 def load_peaks():
@@ -269,7 +269,7 @@ def run_ours(args, cfg):
                 "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES_PER_LAUNCH.get(cfg.name)
-    roof.update({"kernel": "ead_lmhead_kernel", "kernel_us_per_launch": t_kernel * 1e6,
+    roof.update({"kernel": "ead_lmhead_small_kernel" if B <= 16 else "ead_lmhead_kernel", "kernel_us_per_launch": t_kernel * 1e6,
                  "algorithmic_bytes_per_launch": bytes_s.mean(), "flops_per_launch": flops_s.mean(),
                  "peak_source": peaks["source"] + (" (sustained bf16)" if roof["bound"] == "tensor" else ""),
                  "step_frac": (bytes_s.mean() / (t_ms * 1e-3 / K) / 1e9 / peaks["hbm_gbs"]) if roof["bound"] == "hbm"
