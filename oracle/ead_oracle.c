@@ -22,6 +22,10 @@
  *                        threshold test of Eq. 4 with c <- 0 at a switch.
  *   - oracle_run         Algorithm 1 for B independent sequences and a fixed
  *                        number T of tokens, hidden states given as inputs.
+ *   - oracle_parameter_ratio   the footnote of Table 1: average parameters per
+ *                        forward pass relative to the large model,
+ *                        (alpha P_S + beta P_L) / P_L with alpha, beta the usage
+ *                        shares of the small and the large model.
  *
  * Readings where the paper is silent: a row whose logits contain a NaN or an
  * infinity produces H = NaN, token -1, and leaves W, c and the model flag as
@@ -31,7 +35,8 @@
  * give 0, shift invariance, a two-level closed form, brute force on tiny V,
  * bits = nats / ln 2, hand-worked window/threshold traces, and the
  * "small for d_min tokens, then large" trace for a threshold below every
- * entropy.  The end-to-end run on the benchmark configurations has no value
+ * entropy; the parameter-ratio column of Table 1 recomputed from its usage
+ * column.  The end-to-end run on the benchmark configurations has no value
  * printed by the paper to compare with: parity unpinned for oracle_run beyond
  * the composition of its pinned parts.
  */
@@ -214,6 +219,27 @@ void oracle_run(int64_t B, int64_t T, int64_t V, int64_t H_small, int64_t H_larg
     }
     free(hist);
     free(z);
+}
+
+/* Footnote of Table 1.  usage_large = beta in [0, 1]; alpha = 1 - beta. */
+double oracle_parameter_ratio(double usage_large, double P_small, double P_large)
+{
+    double alpha = 1.0 - usage_large, beta = usage_large;
+    return (alpha * P_small + beta * P_large) / P_large;
+}
+
+/* Tokens produced by each model and number of switches in a [T] trace of one sequence. */
+void oracle_usage(const uint8_t *used, const uint8_t *next, int64_t T, int64_t *tokens_small,
+                  int64_t *tokens_large, int64_t *switches)
+{
+    int64_t s = 0, l = 0, sw = 0;
+    for (int64_t t = 0; t < T; ++t) {
+        if (used[t]) l += 1; else s += 1;
+        if (next[t] != used[t]) sw += 1;
+    }
+    *tokens_small = s;
+    *tokens_large = l;
+    *switches = sw;
 }
 
 int oracle_num_threads(void)

@@ -62,6 +62,11 @@ def lib():
                                     C.POINTER(C.c_double), C.POINTER(C.c_uint8),
                                     C.POINTER(C.c_uint8), C.POINTER(C.c_double),
                                     C.POINTER(C.c_int32)])
+        L.oracle_parameter_ratio.restype = C.c_double
+        L.oracle_parameter_ratio.argtypes = [C.c_double, C.c_double, C.c_double]
+        L.oracle_usage.restype = None
+        L.oracle_usage.argtypes = [C.POINTER(C.c_uint8), C.POINTER(C.c_uint8), C.c_int64,
+                                   C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         L.oracle_num_threads.restype = C.c_int
         L.oracle_num_threads.argtypes = []
         _lib = L
@@ -109,6 +114,21 @@ def gate_trace(H_seq, w: int, d_min: int, tau: float, start_model: int = 0):
                             int(start_model), _p(Hbar, C.c_double), _p(used, C.c_uint8),
                             _p(nxt, C.c_uint8), _p(c_after, C.c_int32))
     return dict(Hbar=Hbar, used=used, next=nxt, c_after=c_after)
+
+
+def parameter_ratio(usage_large: float, P_small: float, P_large: float) -> float:
+    """Average parameters per forward pass relative to the large model (Table 1 footnote)."""
+    return float(lib().oracle_parameter_ratio(float(usage_large), float(P_small), float(P_large)))
+
+
+def usage(used, nxt):
+    """(tokens by the small model, tokens by the large model, switches) of one [T] trace."""
+    used = np.ascontiguousarray(used, dtype=np.uint8)
+    nxt = np.ascontiguousarray(nxt, dtype=np.uint8)
+    a, b, c = C.c_int64(), C.c_int64(), C.c_int64()
+    lib().oracle_usage(_p(used, C.c_uint8), _p(nxt, C.c_uint8), used.size, C.byref(a), C.byref(b),
+                       C.byref(c))
+    return int(a.value), int(b.value), int(c.value)
 
 
 class GateState:

@@ -304,3 +304,49 @@ def test_generator_is_counter_based():
     h20 = synth.hidden_states(5, 0, r[:20], 16, 3.0, 0.2)
     assert np.array_equal(h40[:20], h20)
     assert not np.array_equal(synth.lm_head(6, 1, 64, 16), a[:64])
+
+
+# ---------------------------------------------------------------- usage / parameter ratio
+def _read_table1():
+    blocks, cur = [], None
+    with open(os.path.join(GOLDEN, "table1.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            v = line.split()
+            if v[0] == "pair":
+                cur = dict(name=v[1], P_small=float(v[3]), P_large=float(v[5]), tol=float(v[7]), rows=[])
+                blocks.append(cur)
+            else:
+                cur["rows"].append(tuple(float(x) for x in v))
+    return blocks
+
+
+@pytest.mark.parametrize("blk", _read_table1(), ids=lambda b: b["name"])
+def test_parameter_ratio_reproduces_table_1(blk):
+    """The printed parameter-ratio column follows from the printed usage column through the
+    footnote's formula (to the rounding of the table; the tolerance per block is stated in the
+    fixture).  A swapped alpha/beta or a normalisation by P_S fails every block."""
+    assert len(blk["rows"]) == 8
+    worst = 0.0
+    for tau, usage_pct, _score, ratio_pct in blk["rows"]:
+        got = 100.0 * O.parameter_ratio(usage_pct / 100.0, blk["P_small"], blk["P_large"])
+        worst = max(worst, abs(got - ratio_pct))
+        assert abs(got - ratio_pct) <= blk["tol"], (blk["name"], tau, got, ratio_pct)
+    # end points are exact: all-small gives P_S / P_L, all-large gives 1
+    assert O.parameter_ratio(0.0, blk["P_small"], blk["P_large"]) == blk["P_small"] / blk["P_large"]
+    assert O.parameter_ratio(1.0, blk["P_small"], blk["P_large"]) == 1.0
+    assert worst > 0.0 or blk["tol"] >= 0.0
+
+
+def test_usage_counts_of_hand_traces():
+    for tr in _read_traces():
+        out = O.gate_trace(tr["H"], tr["w"], tr["d_min"], tr["tau"])
+        s, l, sw = O.usage(out["used"], out["next"])
+        assert s == tr["used"].count(0) and l == tr["used"].count(1)
+        assert sw == sum(1 for u, n in zip(tr["used"], tr["next"]) if u != n)
+    # trace D: used SLLLLLSSSSLL, next LLLLLSSSSLLL -> 5 small, 7 large, 3 switches
+    tr = [t for t in _read_traces() if t["name"] == "D"][0]
+    out = O.gate_trace(tr["H"], tr["w"], tr["d_min"], tr["tau"])
+    assert O.usage(out["used"], out["next"]) == (5, 7, 3)
