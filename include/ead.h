@@ -155,6 +155,23 @@ size_t ead_state_size(const ead_ctx *ctx);
 int ead_get_state(ead_ctx *ctx, void *host_blob, size_t size);
 int ead_set_state(ead_ctx *ctx, const void *host_blob, size_t size);
 
+/*
+ * Usage accounting since the last ead_reset (the paper's "large model usage" column and the
+ * count of model switches), summed over the B sequences.  Rows with non-finite logits in a
+ * step are not counted for that step.  Waits for the stream.
+ *   counts  host, uint64 [3]: {tokens produced by M_S, tokens produced by M_L, switches}
+ *   per_row host, uint32 [3 * B] or NULL: the same three counters per sequence, row major [3][B]
+ * Errors: EAD_EINVALID_ARG, EAD_ECUDA.
+ */
+int ead_usage(ead_ctx *ctx, uint64_t *counts, uint32_t *per_row);
+
+/*
+ * The footnote of the paper's Table 1: average parameters per forward pass relative to the
+ * large model, (alpha P_S + beta P_L) / P_L, with alpha = tokens_small / total and
+ * beta = tokens_large / total.  Pure host arithmetic; returns NaN if both counts are 0.
+ */
+double ead_parameter_ratio(uint64_t tokens_small, uint64_t tokens_large, double P_small, double P_large);
+
 /* Number of kernels the library has launched through this context so far
  * (graph replays count their kernel nodes). */
 int64_t ead_kernel_launches(const ead_ctx *ctx);

@@ -29,7 +29,7 @@ EAD_STATUS_BAD_COUNT = 0x4
 SYMBOLS = ["ead_create", "ead_step", "ead_run", "ead_run_host", "ead_run_timed", "ead_reset", "ead_status",
            "ead_state_size", "ead_get_state", "ead_set_state", "ead_kernel_launches",
            "ead_launch_info", "ead_destroy", "ead_strerror", "ead_head_entropy_static",
-           "ead_plan_split"]
+           "ead_plan_split", "ead_usage", "ead_parameter_ratio"]
 
 
 class EadConfig(C.Structure):
@@ -86,6 +86,10 @@ def lib() -> C.CDLL:
         L.ead_head_entropy_static.restype = C.c_int
         L.ead_head_entropy_static.argtypes = [vp, vp, C.c_int32, C.c_int32, C.c_int32, i32p, f32p, vp,
                                               C.c_int32, vp]
+        L.ead_usage.restype = C.c_int
+        L.ead_usage.argtypes = [vp, C.POINTER(C.c_uint64), vp]
+        L.ead_parameter_ratio.restype = C.c_double
+        L.ead_parameter_ratio.argtypes = [C.c_uint64, C.c_uint64, C.c_double, C.c_double]
         L.ead_plan_split.restype = C.c_int
         L.ead_plan_split.argtypes = [C.c_int32] * 4 + [C.POINTER(C.c_int32)]
         L.ead_strerror.restype = C.c_char_p
@@ -198,6 +202,19 @@ def ead_head_entropy_static(W, h, B, V, H, tok=None, H_out=None, status=None, de
     _check(lib().ead_head_entropy_static(_ptr(W), _ptr(h), int(B), int(V), int(H), _ptr(tok),
                                          _ptr(H_out), _ptr(status), int(device),
                                          C.c_void_p(int(stream))), "ead_head_entropy_static")
+
+
+def ead_usage(ctx, per_row=None) -> dict:
+    """Tokens produced by each model and switches since the last reset (summed over rows);
+    ``per_row`` may be a uint32 numpy array of shape [3, B] to receive the per-row counters."""
+    a = (C.c_uint64 * 3)()
+    _check(lib().ead_usage(ctx, a, _ptr(per_row)), "ead_usage")
+    return dict(tokens_small=int(a[0]), tokens_large=int(a[1]), switches=int(a[2]))
+
+
+def ead_parameter_ratio(tokens_small, tokens_large, P_small, P_large) -> float:
+    return float(lib().ead_parameter_ratio(int(tokens_small), int(tokens_large), float(P_small),
+                                           float(P_large)))
 
 
 def ead_plan_split(cta, G, n_rows, V) -> dict:

@@ -22,7 +22,7 @@ using namespace ead;
 namespace {
 
 constexpr int kGraphChunk = 32;           // gate steps unrolled in the replayed graph
-constexpr uint32_t kStateMagic = 0x45414431u;   // "EAD1"
+constexpr uint32_t kStateMagic = 0x45414432u;   // "EAD2"
 constexpr size_t kHostStageBytes = 64u << 20;   // per staging buffer of ead_run_host
 
 struct StateHeader {
@@ -79,6 +79,7 @@ struct ead_ctx {
     RunArgs *args = nullptr;
     uint8_t *flag = nullptr;
     int32_t *c = nullptr, *nfill = nullptr, *perm = nullptr, *part_i = nullptr;
+    uint32_t *usage = nullptr;
     float *ring = nullptr, *part_m = nullptr, *part_s = nullptr, *part_t = nullptr;
     uint16_t *hc[2] = {nullptr, nullptr};
     CUtensorMap tmA[2], tmW[2], tmT[2], tmP[2];   // hidden rows; W boxes of 256|128, 16 and 32 rows
@@ -194,6 +195,7 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     gp.c = x->c;
     gp.nfill = x->nfill;
     gp.ring = x->ring;
+    gp.usage = x->usage;
     const int rows_per_block = kGateThreads / 32;
     if (x->small_cols)
         e = launch(ead_merge_gate_wide_kernel, dim3(c.B), dim3(kGateThreads), 0, s, pdl, gp);
@@ -403,6 +405,7 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
         cudaMalloc(&x->flag, B) != cudaSuccess || cudaMalloc(&x->c, 4ull * B) != cudaSuccess ||
         cudaMalloc(&x->nfill, 4ull * B) != cudaSuccess || cudaMalloc(&x->perm, 8ull * B) != cudaSuccess ||
         cudaMalloc(&x->ring, 4ull * B * cfg->w) != cudaSuccess ||
+        cudaMalloc(&x->usage, 12ull * B) != cudaSuccess ||
         cudaMalloc(&x->hc[0], 2ull * Bpad * cfg->H_small) != cudaSuccess ||
         cudaMalloc(&x->hc[1], 2ull * Bpad * cfg->H_large) != cudaSuccess ||
         cudaMalloc(&x->part_m, 4 * np) != cudaSuccess || cudaMalloc(&x->part_s, 4 * np) != cudaSuccess ||
@@ -463,7 +466,8 @@ int ead_reset(ead_ctx *x)
     const ead_config &c = x->cfg;
     const int threads = 256;
     ead_reset_kernel<<<(c.B + threads - 1) / threads, threads, 0, x->stream>>>(x->ctl, x->flag, x->c, x->nfill,
-                                                                              x->ring, c.B, c.w, c.start_model);
+                                                                              x->ring, x->usage, c.B, c.w,
+                                                                              c.start_model);
     x->launches += 1;
     return cudaGetLastError() == cudaSuccess ? EAD_OK : EAD_ECUDA;
 }
@@ -584,7 +588,8 @@ size_t ead_state_size(const ead_ctx *x)
 {
     if (!x) return 0;
     const size_t B = x->cfg.B;
-    return sizeof(StateHeader) + B /*flag*/ + ((4 - B % 4) % 4) + 4 * B /*c*/ + 4 * B /*nfill*/ + 4 * B * x->cfg.w;
+    return sizeof(StateHeader) + B /*flag*/ + ((4 - B % 4) % 4) + 4 * B /*c*/ + 4 * B /*nfill*/ + 12 * B /*usage*/ +
+           4 * B * x->cfg.w;
 }
 
 int ead_get_state(ead_ctx *x, void *blob, size_t size)
@@ -606,6 +611,8 @@ int ead_get_state(ead_ctx *x, void *blob, size_t size)
     p += 4 * B;
     EAD_CUDA(cudaMemcpy(p, x->nfill, 4 * B, cudaMemcpyDeviceToHost));
     p += 4 * B;
+    EAD_CUDA(cudaMemcpy(p, x->usage, 12 * B, cudaMemcpyDeviceToHost));
+    p += 12 * B;
     EAD_CUDA(cudaMemcpy(p, x->ring, 4 * B * x->cfg.w, cudaMemcpyDeviceToHost));
     return EAD_OK;
 }
@@ -630,8 +637,33 @@ int ead_set_state(ead_ctx *x, const void *blob, size_t size)
     p += 4 * B;
     EAD_CUDA(cudaMemcpy(x->nfill, p, 4 * B, cudaMemcpyHostToDevice));
     p += 4 * B;
+    EAD_CUDA(cudaMemcpy(x->usage, p, 12 * B, cudaMemcpyHostToDevice));
+    p += 12 * B;
     EAD_CUDA(cudaMemcpy(x->ring, p, 4 * B * x->cfg.w, cudaMemcpyHostToDevice));
     return EAD_OK;
+}
+
+int ead_usage(ead_ctx *x, uint64_t *counts, uint32_t *per_row)
+{
+    if (!x || !counts) return EAD_EINVALID_ARG;
+    EAD_CUDA(cudaStreamSynchronize(x->stream));
+    const size_t B = x->cfg.B;
+    std::vector<uint32_t> h(3 * B);
+    EAD_CUDA(cudaMemcpy(h.data(), x->usage, 12 * B, cudaMemcpyDeviceToHost));
+    for (int k = 0; k < 3; ++k) {
+        uint64_t s = 0;
+        for (size_t b = 0; b < B; ++b) s += h[k * B + b];
+        counts[k] = s;
+    }
+    if (per_row) memcpy(per_row, h.data(), 12 * B);
+    return EAD_OK;
+}
+
+double ead_parameter_ratio(uint64_t tokens_small, uint64_t tokens_large, double P_small, double P_large)
+{
+    const double total = static_cast<double>(tokens_small) + static_cast<double>(tokens_large);
+    const double alpha = static_cast<double>(tokens_small) / total, beta = static_cast<double>(tokens_large) / total;
+    return (alpha * P_small + beta * P_large) / P_large;
 }
 
 int64_t ead_kernel_launches(const ead_ctx *x) { return x ? x->launches : 0; }
@@ -670,7 +702,7 @@ void ead_destroy(ead_ctx *x)
     if (x->g_chunk) cudaGraphExecDestroy(x->g_chunk);
     if (x->cap_stream) cudaStreamDestroy(x->cap_stream);
     void *bufs[] = {x->ctl, x->args, x->flag, x->c, x->nfill, x->perm, x->ring, x->hc[0], x->hc[1],
-                    x->part_m, x->part_s, x->part_t, x->part_i};
+                    x->part_m, x->part_s, x->part_t, x->part_i, x->usage};
     for (void *b : bufs)
         if (b) cudaFree(b);
     cudaGetLastError();

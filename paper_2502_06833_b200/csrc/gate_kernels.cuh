@@ -23,7 +23,7 @@ __global__ void ead_set_args_kernel(RunArgs *dst, RunArgs a, const StepCtl *ctl)
 }
 
 __global__ void ead_reset_kernel(StepCtl *ctl, uint8_t *flag, int32_t *c, int32_t *nfill, float *ring,
-                                 int B, int w, int start_model)
+                                 uint32_t *usage, int B, int w, int start_model)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i == 0) {
@@ -36,6 +36,7 @@ __global__ void ead_reset_kernel(StepCtl *ctl, uint8_t *flag, int32_t *c, int32_
         flag[i] = static_cast<uint8_t>(start_model);
         c[i] = 0;
         nfill[i] = 0;
+        usage[i] = usage[B + i] = usage[2 * B + i] = 0u;
     }
     for (int k = i; k < B * w; k += gridDim.x * blockDim.x) ring[k] = 0.f;
 }
@@ -112,12 +113,34 @@ struct GateParams {
     int32_t *c;
     int32_t *nfill;
     float *ring;
+    uint32_t *usage;           // [3][B]: tokens by the small model, by the large model, switches
 };
 
 // Everything after the merge for one compacted row (executed by one thread): Eq. 2 in the
 // fused form, then the tail of Algorithm 1's loop body (window, counter, Eq. 4), state update
 // and outputs scattered back to the caller's row.
-__device__ __forceinline__ void finish_row(const GateParams &p, int m, int r, const Partial &acc, int t_step)
+// State of one sequence as finish_row needs it; `ring` points at the w window slots (global or a
+// shared-memory copy, in which case the new entropy is also written through to `ring_global`).
+struct RowState {
+    int b, model, nf, c, run_base;
+    const float *ring;
+    float *ring_global;
+};
+
+__device__ __forceinline__ RowState load_row_state(const GateParams &p, int m, int r)
+{
+    RowState st;
+    st.b = p.perm[m * p.B + r];
+    st.model = p.flag[st.b];
+    st.nf = p.nfill[st.b];
+    st.c = p.c[st.b];
+    st.run_base = p.args->run_base;
+    st.ring_global = p.ring + static_cast<size_t>(st.b) * p.w;
+    st.ring = st.ring_global;
+    return st;
+}
+
+__device__ __forceinline__ void finish_row(const GateParams &p, const RowState &st, const Partial &acc, int t_step)
 {
     // ---- Eq. 2 in the fused form  H = ln Z - E_p[z] = ln s - t / (s log2 e)   (nats)
     float H = logf(acc.s) - acc.t / (acc.s * kLog2e);
@@ -125,9 +148,9 @@ __device__ __forceinline__ void finish_row(const GateParams &p, int m, int r, co
     if (H < 0.f) H = 0.f;                         // rounding can leave -1e-7 for a one-hot row
     if (p.unit == 1) H *= kLog2e;                 // bits, as Eq. 2 is printed
 
-    const int b = p.perm[m * p.B + r];
-    const size_t o = static_cast<size_t>(t_step - p.args->run_base) * p.B + b;
-    int model = p.flag[b];
+    const int b = st.b;
+    const size_t o = static_cast<size_t>(t_step - st.run_base) * p.B + b;
+    int model = st.model;
     if (!finite) {
         // non-finite logits: report, leave window, counter and model untouched
         atomicOr(&p.ctl->status, kStatusNonFinite);
@@ -139,16 +162,16 @@ __device__ __forceinline__ void finish_row(const GateParams &p, int m, int r, co
         return;
     }
     // ---- Algorithm 1: append H_t to W; mean of the last w entries (those present)
-    int nf = p.nfill[b];
-    float *ring = p.ring + static_cast<size_t>(b) * p.w;
-    ring[nf % p.w] = H;
+    int nf = st.nf;
+    const int slot = nf % p.w;
+    st.ring_global[slot] = H;
     nf += 1;
     const int cnt = nf < p.w ? nf : p.w;
     float sum = 0.f;
-    for (int k = 0; k < cnt; ++k) sum += ring[k];
+    for (int k = 0; k < cnt; ++k) sum += (k == slot) ? H : st.ring[k];     // slot order, as stored
     const float Hbar = sum / static_cast<float>(cnt);
     // ---- c <- c + 1; Eq. 4
-    int c = p.c[b] + 1;
+    int c = st.c + 1;
     const int used = model;
     if (c >= p.d_min) {
         if (model == 0 && Hbar > p.tau) { model = 1; c = 0; }
@@ -157,6 +180,8 @@ __device__ __forceinline__ void finish_row(const GateParams &p, int m, int r, co
     p.nfill[b] = nf;
     p.c[b] = c;
     p.flag[b] = static_cast<uint8_t>(model);
+    p.usage[used * p.B + b] += 1u;                     // this row is owned by this thread: no atomics
+    if (model != used) p.usage[2 * p.B + b] += 1u;
     if (p.args->tok) p.args->tok[o] = acc.idx;
     if (p.args->H) p.args->H[o] = H;
     if (p.args->Hbar) p.args->Hbar[o] = Hbar;
@@ -208,7 +233,7 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const Gate
         acc = merge_partial(acc, q);
     }
     acc = warp_merge(acc);
-    if (lane == 0) finish_row(p, m, r, acc, t_step);
+    if (lane == 0) finish_row(p, load_row_state(p, m, r), acc, t_step);
 }
 
 // One block per compacted row: the 4 G partials of the small-batch kernel.  Thread t folds slots t, t + 256, ... in ascending order, then lanes, then warps:
@@ -216,19 +241,33 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const Gate
 __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_wide_kernel(const GateParams p)
 {
     __shared__ Partial wsum[kGateThreads / 32];
+    __shared__ float ring_sh[64];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int i = blockIdx.x;
     griddep_launch_dependents();
-    griddep_wait();                              // partials of the LM-head kernel
+    // This kernel is released as soon as the LM-head kernel is past its own dependency wait,
+    // i.e. after the compaction kernel has finished: row counts, permutation and the state of
+    // the previous step are final, and loading them here hides their latency behind the
+    // LM-head kernel.  Only the partials need the wait below.
     const int n0 = p.ctl->n[0], n1 = p.ctl->n[1];
     const int t_step = p.ctl->cur_t;
+    const bool live = i < p.B && n0 + n1 == p.B;
+    const int m = i < n0 ? 0 : 1;
+    const int r = m ? i - n0 : i;
+    RowState st{};
+    if (live) {
+        if (threadIdx.x == 0) st = load_row_state(p, m, r);
+        const int b = p.perm[m * p.B + r];
+        if (threadIdx.x < p.w) ring_sh[threadIdx.x] = p.ring[static_cast<size_t>(b) * p.w + threadIdx.x];
+    }
+    st.ring = ring_sh;
+    __syncthreads();
+    griddep_wait();                              // partials of the LM-head kernel
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         if (n0 + n1 != p.B) atomicOr(&p.ctl->status, kStatusBadCount);
         p.ctl->step = t_step + 1;
     }
-    if (i >= p.B || n0 + n1 != p.B) return;
-    const int m = i < n0 ? 0 : 1;
-    const int r = m ? i - n0 : i;
+    if (!live) return;
     const size_t base = (static_cast<size_t>(m) * p.B + r) * p.slots_stride;
     Partial acc{kNegSentinel, 0.f, 0.f, 0x7fffffff};
     for (int s = threadIdx.x; s < p.n_slots; s += kGateThreads) {
@@ -242,7 +281,7 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_wide_kernel(const
         acc = wsum[0];
 #pragma unroll
         for (int k = 1; k < kGateThreads / 32; ++k) acc = merge_partial(acc, wsum[k]);
-        finish_row(p, m, r, acc, t_step);
+        finish_row(p, st, acc, t_step);
     }
 }
 

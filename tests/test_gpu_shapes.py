@@ -197,3 +197,26 @@ def test_largest_batch_and_zero_steps():
         g.E.ead_run(g.ctx, 0, 16, 16)                  # T = 0 is a no-op
         out = g.run(wl.h_small, wl.h_large, "run")
     compare(out, ora, cfg.tau)
+
+
+def test_usage_counters_follow_the_trace_and_survive_a_checkpoint():
+    cfg = _cfg(B=6, V=1500, T=40, tau=_mid_tau(1500))
+    wl = synth.Workload(cfg)
+    ora = _oracle(cfg, wl)
+    want = [O.usage(ora["used"][:, b], ora["next"][:, b]) for b in range(cfg.B)]
+    per_row = np.zeros((3, cfg.B), dtype=np.uint32)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        g.run(wl.h_small[:25], wl.h_large[:25], "run")
+        blob = g.E.ead_get_state(g.ctx)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        g.E.ead_set_state(g.ctx, blob)
+        g.run(wl.h_small[25:], wl.h_large[25:], "run")
+        tot = g.E.ead_usage(g.ctx, per_row)
+        ratio = g.E.ead_parameter_ratio(tot["tokens_small"], tot["tokens_large"], 1.0, 3.0)
+        g.E.ead_reset(g.ctx)
+        assert g.E.ead_usage(g.ctx) == dict(tokens_small=0, tokens_large=0, switches=0)
+    assert per_row.T.tolist() == [list(w) for w in want]
+    assert tot == dict(tokens_small=sum(w[0] for w in want), tokens_large=sum(w[1] for w in want),
+                       switches=sum(w[2] for w in want))
+    assert tot["tokens_small"] + tot["tokens_large"] == cfg.B * cfg.T
+    assert ratio == pytest.approx(O.parameter_ratio(ora["used"].mean(), 1.0, 3.0), rel=1e-12)

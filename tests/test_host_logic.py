@@ -143,3 +143,12 @@ def test_aggregation_over_two_ranks_takes_the_slowest(tmp_path):
     res = subprocess.run(cmd, capture_output=True, text=True, timeout=240)
     assert res.returncode == 0, res.stdout + res.stderr
     assert res.stdout.count("ok") == 2
+
+
+def test_parameter_ratio_matches_the_table_footnote(E):
+    """Host arithmetic of the library against two rows of the paper's Table 1 (Qwen 14B vs
+    1.5B at 25.6 % usage -> 33.6 %; LLaMA 3B vs 1B at 16.0 % -> 44.0 %) and the end points."""
+    assert 100 * E.ead_parameter_ratio(744, 256, 1.5, 14) == pytest.approx(33.6, abs=0.1)
+    assert 100 * E.ead_parameter_ratio(84, 16, 1, 3) == pytest.approx(44.0, abs=0.05)
+    assert E.ead_parameter_ratio(10, 0, 3, 11) == pytest.approx(3 / 11)
+    assert E.ead_parameter_ratio(0, 10, 3, 11) == 1.0
