@@ -22,6 +22,14 @@
  *                        threshold test of Eq. 4 with c <- 0 at a switch.
  *   - oracle_run         Algorithm 1 for B independent sequences and a fixed
  *                        number T of tokens, hidden states given as inputs.
+ *   - oracle_sample      the sampling lines of Algorithm 1: l' = l / T, p' =
+ *                        softmax(l'), token ~ p'.  The draw is realised as the
+ *                        arg max of l'_i + g_i with independent standard Gumbel
+ *                        g_i = -ln(-ln u_i) (an exact sampler of p'), the
+ *                        uniforms u_i coming from Philox4x32-10 (Salmon, Moraes,
+ *                        Dror, Shaw, SC'11) keyed by (seed) and counted by
+ *                        (vocabulary index / 4, step, row): the same stream the
+ *                        CUDA path implements from the same published definition.
  *   - oracle_parameter_ratio   the footnote of Table 1: average parameters per
  *                        forward pass relative to the large model,
  *                        (alpha P_S + beta P_L) / P_L with alpha, beta the usage
@@ -125,6 +133,66 @@ int64_t oracle_greedy(const double *z, int64_t V, double *gap_out)
     return best;
 }
 
+/* ---- Philox4x32-10 as published: 10 rounds of two 32x32 -> 64 multiplies with the
+ *      constants 0xD2511F53, 0xCD9E8D57 and the key bumped by 0x9E3779B9, 0xBB67AE85. */
+void oracle_philox4x32(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int r = 0; r < 10; ++r) {
+        uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* Uniform in (0, 1) for vocabulary entry i of sequence `row` at its `step`-th token:
+ * the top 23 bits k of word (i mod 4) of block (i / 4), as (2k + 1) / 2^24 (an odd
+ * multiple of 2^-24: exact in float32 and float64, never 0 or 1). */
+double oracle_uniform(uint64_t seed, int64_t row, int64_t step, int64_t i)
+{
+    uint32_t ctr[4] = {(uint32_t)(i >> 2), (uint32_t)step, (uint32_t)row, 0u};
+    uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    uint32_t out[4];
+    oracle_philox4x32(ctr, key, out);
+    uint32_t k = out[i & 3] >> 9;
+    return (double)(2u * k + 1u) / 16777216.0;
+}
+
+/* Sampling lines of Algorithm 1 at temperature T > 0 (see the header).  Returns the
+ * token; gap_out receives the difference of the two largest perturbed values. */
+int64_t oracle_sample(const double *z, int64_t V, double T, uint64_t seed, int64_t row,
+                      int64_t step, double *gap_out)
+{
+    if (V <= 0 || !all_finite(z, V)) {
+        if (gap_out) *gap_out = NAN;
+        return -1;
+    }
+    int64_t best = -1;
+    double best_v = -INFINITY, second = -INFINITY;
+    for (int64_t i = 0; i < V; ++i) {
+        double lp = z[i] / T;                                /* l' = l / T          */
+        double g = -log(-log(oracle_uniform(seed, row, step, i)));
+        double v = lp + g;                                   /* arg max = draw from softmax(l') */
+        if (v > best_v) {
+            second = best_v;
+            best_v = v;
+            best = i;
+        } else if (v > second) {
+            second = v;
+        }
+    }
+    if (gap_out) *gap_out = (V > 1) ? best_v - second : INFINITY;
+    return best;
+}
+
 /*
  * One pass through the tail of Algorithm 1's loop body for one sequence.
  *   hist     entropy window W as the paper keeps it: an append-only list
@@ -174,7 +242,7 @@ void oracle_gate_trace(const double *H, int64_t T, int32_t w, int32_t d_min, dou
 }
 
 /*
- * Algorithm 1 with greedy selection for the rows listed in `rows` (n_rows of
+ * Algorithm 1 (greedy for temperature 0, sampled otherwise) for the rows listed in `rows` (n_rows of
  * them, indices into [0, B)) and T tokens.  Inputs are bf16 bit patterns:
  * W_small [V, H_small], W_large [V, H_large], h_small [T, B, H_small],
  * h_large [T, B, H_large].  Outputs are [T, n_rows], row k of an output
@@ -189,7 +257,7 @@ void oracle_run(int64_t B, int64_t T, int64_t V, int64_t H_small, int64_t H_larg
                 const uint16_t *h_small, const uint16_t *h_large,
                 const int64_t *rows, int64_t n_rows,
                 int32_t *tok, double *H, double *Hbar, uint8_t *used, uint8_t *next,
-                double *gap, int32_t *c_after)
+                double *gap, int32_t *c_after, double temperature, uint64_t seed)
 {
     double *z = (double *)malloc((size_t)V * sizeof(double));
     double *hist = (double *)malloc((size_t)(T > 0 ? T : 1) * sizeof(double));
@@ -207,7 +275,10 @@ void oracle_run(int64_t B, int64_t T, int64_t V, int64_t H_small, int64_t H_larg
                 oracle_logits(W_large, V, H_large, h_large + (t * B + b) * H_large, z);
             double Ht = oracle_entropy(z, V, unit, NULL);
             double g;
-            int64_t tk = oracle_greedy(z, V, &g);
+            /* the entropy above is taken before any temperature scaling; the token is the
+               arg max (temperature 0) or a draw from softmax(l / T) */
+            int64_t tk = temperature > 0.0 ? oracle_sample(z, V, temperature, seed, b, t, &g)
+                                           : oracle_greedy(z, V, &g);
             double Hb = oracle_gate_step(hist, &n, &c, &model, Ht, w, d_min, tau);
             if (tok) tok[o] = (int32_t)tk;
             if (H) H[o] = Ht;

@@ -61,7 +61,14 @@ def lib():
                                  + [C.POINTER(C.c_int32), C.POINTER(C.c_double),
                                     C.POINTER(C.c_double), C.POINTER(C.c_uint8),
                                     C.POINTER(C.c_uint8), C.POINTER(C.c_double),
-                                    C.POINTER(C.c_int32)])
+                                    C.POINTER(C.c_int32), C.c_double, C.c_uint64])
+        L.oracle_philox4x32.restype = None
+        L.oracle_philox4x32.argtypes = [C.POINTER(C.c_uint32)] * 3
+        L.oracle_uniform.restype = C.c_double
+        L.oracle_uniform.argtypes = [C.c_uint64, C.c_int64, C.c_int64, C.c_int64]
+        L.oracle_sample.restype = C.c_int64
+        L.oracle_sample.argtypes = [C.POINTER(C.c_double), C.c_int64, C.c_double, C.c_uint64,
+                                    C.c_int64, C.c_int64, C.POINTER(C.c_double)]
         L.oracle_parameter_ratio.restype = C.c_double
         L.oracle_parameter_ratio.argtypes = [C.c_double, C.c_double, C.c_double]
         L.oracle_usage.restype = None
@@ -147,8 +154,30 @@ class GateState:
                                             int(w), int(d_min), float(tau)))
 
 
+def philox4x32(ctr, key):
+    c = (C.c_uint32 * 4)(*[int(x) & 0xFFFFFFFF for x in ctr])
+    k = (C.c_uint32 * 2)(*[int(x) & 0xFFFFFFFF for x in key])
+    o = (C.c_uint32 * 4)()
+    lib().oracle_philox4x32(c, k, o)
+    return [int(x) for x in o]
+
+
+def uniform(seed: int, row: int, step: int, i: int) -> float:
+    return float(lib().oracle_uniform(int(seed), int(row), int(step), int(i)))
+
+
+def sample(z, temperature: float, seed: int, row: int, step: int):
+    """(token drawn from softmax(z / T), gap between the two largest perturbed values)."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    gap = C.c_double()
+    tok = lib().oracle_sample(_p(z, C.c_double), z.size, float(temperature), int(seed), int(row),
+                              int(step), C.byref(gap))
+    return int(tok), float(gap.value)
+
+
 def run(W_small, W_large, h_small, h_large, *, w: int, d_min: int, tau: float, unit: int = 0,
-        start_model: int = 0, rows=None, T: int | None = None):
+        start_model: int = 0, rows=None, T: int | None = None, temperature: float = 0.0,
+        seed: int = 0):
     """Algorithm 1 (greedy) on bf16 bit-pattern inputs.
 
     ``h_small``/``h_large`` are ``[T, B, H]`` uint16; ``rows`` selects which of
@@ -180,7 +209,7 @@ def run(W_small, W_large, h_small, h_large, *, w: int, d_min: int, tau: float, u
                      _p(out["tok"], C.c_int32), _p(out["H"], C.c_double),
                      _p(out["Hbar"], C.c_double), _p(out["used"], C.c_uint8),
                      _p(out["next"], C.c_uint8), _p(out["gap"], C.c_double),
-                     _p(out["c_after"], C.c_int32))
+                     _p(out["c_after"], C.c_int32), float(temperature), int(seed))
     return out
 
 

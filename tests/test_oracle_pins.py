@@ -350,3 +350,76 @@ def test_usage_counts_of_hand_traces():
     tr = [t for t in _read_traces() if t["name"] == "D"][0]
     out = O.gate_trace(tr["H"], tr["w"], tr["d_min"], tr["tau"])
     assert O.usage(out["used"], out["next"]) == (5, 7, 3)
+
+
+# ---------------------------------------------------------------- sampling (Algorithm 1, sampling lines)
+def test_philox_known_answers():
+    """Known-answer vectors of Philox4x32-10 published with the Random123 library."""
+    assert O.philox4x32([0, 0, 0, 0], [0, 0]) == [0x6627e8d5, 0xe169c58d, 0xbc57ac4c, 0x9b00dbd8]
+    assert O.philox4x32([0xffffffff] * 4, [0xffffffff] * 2) == [0x408f276d, 0x41c83b0e, 0xa20bc7c6,
+                                                                 0x6d5451fd]
+    assert O.philox4x32([0x243f6a88, 0x85a308d3, 0x13198a2e, 0x03707344],
+                        [0xa4093822, 0x299f31d0]) == [0xd16cfe09, 0x94fdcceb, 0x5001e420, 0x24126ea1]
+
+
+def test_uniform_is_an_odd_multiple_of_2_pow_minus_24_and_flat():
+    u = np.array([O.uniform(9, 3, 5, i) for i in range(20000)])
+    k = u * 2 ** 24
+    assert np.all(k == np.round(k)) and np.all(k.astype(np.int64) % 2 == 1)
+    assert 0.0 < u.min() and u.max() < 1.0
+    assert np.array_equal(u.astype(np.float32).astype(np.float64), u)      # exact in float32
+    hist = np.histogram(u, bins=20, range=(0, 1))[0]
+    chi2 = ((hist - 1000.0) ** 2 / 1000.0).sum()
+    assert chi2 < 50.0                                                     # 19 d.o.f.: p ~ 1e-4
+    # different (row, step) give different streams; blocks of 4 indices share one Philox call
+    assert O.uniform(9, 3, 5, 0) != O.uniform(9, 3, 6, 0) != O.uniform(9, 4, 5, 0)
+    w = O.philox4x32([1, 5, 3, 0], [9, 0])
+    assert [O.uniform(9, 3, 5, 4 + j) for j in range(4)] == [(2 * (x >> 9) + 1) / 2 ** 24 for x in w]
+
+
+def test_sampled_tokens_follow_softmax_of_logits_over_temperature():
+    """Draws are distributed as p' = softmax(l / T) (chi-square against the exact p'), and an
+    inverse-CDF sampler fed with independent uniforms agrees with that distribution too."""
+    rng = np.random.default_rng(21)
+    z = rng.normal(0, 1.5, 6)
+    for T in (0.5, 1.0, 2.0):
+        p = scipy.special.softmax(z / T)
+        n = 20000
+        counts = np.bincount([O.sample(z, T, 77, 0, step)[0] for step in range(n)], minlength=6)
+        chi2 = ((counts - n * p) ** 2 / (n * p)).sum()
+        assert chi2 < 25.0, (T, counts, n * p)                            # 5 d.o.f.: p ~ 1e-4
+        inv = np.searchsorted(np.cumsum(p), rng.random(n))
+        chi2_inv = ((np.bincount(inv, minlength=6) - n * p) ** 2 / (n * p)).sum()
+        assert chi2_inv < 25.0
+    # temperature -> 0 approaches the arg max; a huge temperature approaches uniform
+    cold = [O.sample(z, 1e-3, 5, 0, s)[0] for s in range(200)]
+    assert set(cold) == {int(np.argmax(z))}
+    hot = np.bincount([O.sample(z, 1e6, 5, 0, s)[0] for s in range(6000)], minlength=6)
+    assert hot.min() > 800
+
+
+def test_sample_is_argmax_of_perturbed_scaled_logits():
+    rng = np.random.default_rng(22)
+    z = rng.normal(0, 2, 50)
+    for step in range(20):
+        T = 0.7
+        v = z / T - np.log(-np.log([O.uniform(3, 11, step, i) for i in range(50)]))
+        tok, gap = O.sample(z, T, 3, 11, step)
+        order = np.argsort(-v)
+        assert tok == order[0] and gap == pytest.approx(v[order[0]] - v[order[1]], abs=1e-12)
+
+
+def test_run_with_temperature_keeps_entropy_and_switches_of_the_greedy_run():
+    """Entropy is taken before temperature scaling, and hidden states are inputs here, so only
+    the token column changes when sampling is switched on."""
+    r, Ws, Wl, hs, hl = _tiny_inputs()
+    a = O.run(Ws, Wl, hs, hl, w=3, d_min=2, tau=4.6)
+    b = O.run(Ws, Wl, hs, hl, w=3, d_min=2, tau=4.6, temperature=1.0, seed=5)
+    for k in ("H", "Hbar", "used", "next"):
+        assert np.array_equal(a[k], b[k])
+    assert (a["tok"] != b["tok"]).mean() > 0.3
+    T, B = r.shape
+    for t in (0, 7, T - 1):
+        for bb in range(B):
+            z = O.logits(Ws, hs[t, bb]) if b["used"][t, bb] == 0 else O.logits(Wl, hl[t, bb])
+            assert b["tok"][t, bb] == O.sample(z, 1.0, 5, bb, t)[0]
