@@ -69,6 +69,8 @@ typedef struct ead_config {
     int32_t start_model; /* model of the first token; Algorithm 1 starts on 0 (small)         */
     int32_t device;      /* CUDA device ordinal                                               */
     void   *stream;      /* cudaStream_t to enqueue on (borrowed); NULL = legacy default      */
+    float   temperature; /* T of Algorithm 1's sampling lines; 0 = greedy (arg max)           */
+    uint64_t seed;       /* seed of the sampling random stream (used when temperature > 0)    */
 } ead_config;
 
 /*
@@ -88,8 +90,13 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
  *   h_small     dev, bf16 [B, H_small]: final hidden state of M_S per sequence
  *   h_large     dev, bf16 [B, H_large]: the same for M_L
  *               Only the row of the model that is active for a sequence is read.
- *   tok         dev, int32 [B]: greedy token (lowest index among equal maxima; -1 for a
- *               row with non-finite logits)
+ *   tok         dev, int32 [B]: next token: with cfg.temperature = 0 the arg max (lowest index
+ *               among equal maxima); with cfg.temperature = T > 0 a draw from softmax(l / T),
+ *               realised as arg max of l_i / T + g_i with standard Gumbel g_i = -ln(-ln u_i),
+ *               u_i = (2k + 1) / 2^24, k = top 23 bits of word (i mod 4) of
+ *               Philox4x32-10(counter = {i / 4, step, row, 0}, key = seed), step = number of
+ *               gate steps of the context since the last reset.  -1 for a row with
+ *               non-finite logits
  *   H           dev, float [B]: entropy of Eq. 2 in cfg.unit
  *   Hbar        dev, float [B]: rolling mean of Eq. 3 after this token
  *   model_used  dev, uint8 [B]: model that produced this token

@@ -78,7 +78,8 @@ struct ead_ctx {
     StepCtl *ctl = nullptr;
     RunArgs *args = nullptr;
     uint8_t *flag = nullptr;
-    int32_t *c = nullptr, *nfill = nullptr, *perm = nullptr, *part_i = nullptr;
+    int32_t *c = nullptr, *nfill = nullptr, *perm = nullptr, *part_i = nullptr, *part_ki = nullptr;
+    float *part_k = nullptr;
     uint32_t *usage = nullptr;
     float *ring = nullptr, *part_m = nullptr, *part_s = nullptr, *part_t = nullptr;
     uint16_t *hc[2] = {nullptr, nullptr};
@@ -155,14 +156,25 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     lp.part_s = x->part_s;
     lp.part_t = x->part_t;
     lp.part_i = x->part_i;
+    lp.sampling = c.temperature > 0.f ? 1 : 0;
+    lp.inv_temperature = c.temperature > 0.f ? 1.f / c.temperature : 0.f;
+    lp.seed_lo = static_cast<uint32_t>(c.seed);
+    lp.seed_hi = static_cast<uint32_t>(c.seed >> 32);
+    lp.part_k = x->part_k;
+    lp.part_ki = x->part_ki;
+    lp.perm = x->perm;
     const dim3 lgrid(x->G), lblock(kLmheadThreads);
-#define EAD_LAUNCH_SMALL(NB)                                                                                  \
-    e = launch(ead_lmhead_small_kernel<NB>, lgrid, lblock, x->smem_bytes, s, pdl, x->tmA[0], x->tmA[1], x->tmW[0], \
-               x->tmW[1], x->tmP[0], x->tmP[1], lp)
+#define EAD_LAUNCH_SMALL(NB)                                                                                   \
+    e = lp.sampling ? launch(ead_lmhead_small_kernel<NB, true>, lgrid, lblock, x->smem_bytes, s, pdl, x->tmA[0],  \
+                             x->tmA[1], x->tmW[0], x->tmW[1], x->tmP[0], x->tmP[1], lp)                        \
+                    : launch(ead_lmhead_small_kernel<NB, false>, lgrid, lblock, x->smem_bytes, s, pdl, x->tmA[0], \
+                             x->tmA[1], x->tmW[0], x->tmW[1], x->tmP[0], x->tmP[1], lp)
     switch (x->small_cols) {
         case 0:
-            e = launch(ead_lmhead_kernel, lgrid, lblock, x->smem_bytes, s, pdl, x->tmA[0], x->tmA[1], x->tmW[0],
-                       x->tmW[1], x->tmT[0], x->tmT[1], lp);
+            e = lp.sampling ? launch(ead_lmhead_kernel<true>, lgrid, lblock, x->smem_bytes, s, pdl, x->tmA[0], x->tmA[1],
+                                     x->tmW[0], x->tmW[1], x->tmT[0], x->tmT[1], lp)
+                            : launch(ead_lmhead_kernel<false>, lgrid, lblock, x->smem_bytes, s, pdl, x->tmA[0], x->tmA[1],
+                                     x->tmW[0], x->tmW[1], x->tmT[0], x->tmT[1], lp);
             break;
         case 1: EAD_LAUNCH_SMALL(1); break;
         case 2: EAD_LAUNCH_SMALL(2); break;
@@ -190,6 +202,9 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     gp.part_s = x->part_s;
     gp.part_t = x->part_t;
     gp.part_i = x->part_i;
+    gp.sampling = c.temperature > 0.f ? 1 : 0;
+    gp.part_k = x->part_k;
+    gp.part_ki = x->part_ki;
     gp.perm = x->perm;
     gp.flag = x->flag;
     gp.c = x->c;
@@ -348,7 +363,8 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     if (!cfg || !W_small || !W_large || !out) return EAD_EINVALID_ARG;
     *out = nullptr;
     if (cfg->B < 1 || cfg->B > 4096 || cfg->V < 1 || cfg->H_small < 8 || cfg->H_large < 8 || cfg->w < 1 ||
-        cfg->w > 64 || (cfg->unit != 0 && cfg->unit != 1) || (cfg->start_model != 0 && cfg->start_model != 1))
+        cfg->w > 64 || (cfg->unit != 0 && cfg->unit != 1) || (cfg->start_model != 0 && cfg->start_model != 1) ||
+        !(cfg->temperature >= 0.f) || !(cfg->temperature < 3.0e38f))
         return EAD_EINVALID_ARG;
     if (cfg->H_small % 8 || cfg->H_large % 8 || !aligned16(W_small) || !aligned16(W_large)) return EAD_EALIGNMENT;
 
@@ -409,7 +425,8 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
         cudaMalloc(&x->hc[0], 2ull * Bpad * cfg->H_small) != cudaSuccess ||
         cudaMalloc(&x->hc[1], 2ull * Bpad * cfg->H_large) != cudaSuccess ||
         cudaMalloc(&x->part_m, 4 * np) != cudaSuccess || cudaMalloc(&x->part_s, 4 * np) != cudaSuccess ||
-        cudaMalloc(&x->part_t, 4 * np) != cudaSuccess || cudaMalloc(&x->part_i, 4 * np) != cudaSuccess)
+        cudaMalloc(&x->part_t, 4 * np) != cudaSuccess || cudaMalloc(&x->part_i, 4 * np) != cudaSuccess ||
+        cudaMalloc(&x->part_k, 4 * np) != cudaSuccess || cudaMalloc(&x->part_ki, 4 * np) != cudaSuccess)
         return fail(EAD_ECUDA);
     cudaMemsetAsync(x->ctl, 0, sizeof(StepCtl), x->stream);
     cudaMemsetAsync(x->args, 0, sizeof(RunArgs), x->stream);
@@ -420,6 +437,8 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     cudaMemsetAsync(x->part_s, 0, 4 * np, x->stream);
     cudaMemsetAsync(x->part_t, 0, 4 * np, x->stream);
     cudaMemsetAsync(x->part_i, 0, 4 * np, x->stream);
+    cudaMemsetAsync(x->part_k, 0, 4 * np, x->stream);
+    cudaMemsetAsync(x->part_ki, 0, 4 * np, x->stream);
 
     const uint32_t wbox = static_cast<uint32_t>(
         std::min(x->small_cols ? kSmallTileRows : kTileN, (cfg->V + kUnit - 1) / kUnit * kUnit));
@@ -434,9 +453,18 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     // the attribute belongs to the kernel on this device, not to the context: ask for the
     // device maximum so that contexts with different stage counts can coexist
     const void *lmhead_kernels[] = {
-        reinterpret_cast<const void *>(ead_lmhead_kernel),          reinterpret_cast<const void *>(ead_lmhead_small_kernel<1>),
-        reinterpret_cast<const void *>(ead_lmhead_small_kernel<2>), reinterpret_cast<const void *>(ead_lmhead_small_kernel<4>),
-        reinterpret_cast<const void *>(ead_lmhead_small_kernel<8>), reinterpret_cast<const void *>(ead_lmhead_small_kernel<16>)};
+        reinterpret_cast<const void *>(ead_lmhead_kernel<false>),
+        reinterpret_cast<const void *>(ead_lmhead_kernel<true>),
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<1, false>),
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<2, false>),
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<4, false>),
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<8, false>),
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<16, false>),
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<1, true>),
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<2, true>),
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<4, true>),
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<8, true>),
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<16, true>)};
     for (const void *k : lmhead_kernels) {
         cudaFuncAttributes fa;
         if (cudaFuncGetAttributes(&fa, k) != cudaSuccess) return fail(EAD_ECUDA);
@@ -702,7 +730,7 @@ void ead_destroy(ead_ctx *x)
     if (x->g_chunk) cudaGraphExecDestroy(x->g_chunk);
     if (x->cap_stream) cudaStreamDestroy(x->cap_stream);
     void *bufs[] = {x->ctl, x->args, x->flag, x->c, x->nfill, x->perm, x->ring, x->hc[0], x->hc[1],
-                    x->part_m, x->part_s, x->part_t, x->part_i, x->usage};
+                    x->part_m, x->part_s, x->part_t, x->part_i, x->usage, x->part_k, x->part_ki};
     for (void *b : bufs)
         if (b) cudaFree(b);
     cudaGetLastError();
@@ -819,7 +847,7 @@ int static_device_setup(int device, StaticDevice **out)
         if (!ptr) return EAD_ECUDA;
         EAD_CUDA(cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, device));
         EAD_CUDA(cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device));
-        EAD_CUDA(cudaFuncSetAttribute(ead_lmhead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, d.smem_optin));
+        EAD_CUDA(cudaFuncSetAttribute(ead_lmhead_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.smem_optin));
         d.scratch = static_cast<StaticScratch *>(ptr);
         d.ready = true;
     }
@@ -876,7 +904,7 @@ extern "C" int ead_head_entropy_static(const void *W, const void *h, int32_t B, 
     lp.part_s = sc->part_s;
     lp.part_t = sc->part_t;
     lp.part_i = sc->part_i;
-    ead_lmhead_kernel<<<G, kLmheadThreads, smem_bytes, s>>>(tmA, tmA, tmW, tmW, tmT, tmT, lp);
+    ead_lmhead_kernel<false><<<G, kLmheadThreads, smem_bytes, s>>>(tmA, tmA, tmW, tmW, tmT, tmT, lp);
     const int rows_per_block = kGateThreads / 32;
     ead_static_merge_kernel<<<(B + rows_per_block - 1) / rows_per_block, kGateThreads, 0, s>>>(sc, B, G, tok, H_out,
                                                                                              status);

@@ -98,6 +98,43 @@ __device__ __forceinline__ Partial merge_partial(const Partial &a, const Partial
     return r;
 }
 
+// A sampled token candidate: largest perturbed logit and its column; equal values keep the
+// lower column.
+struct Draw {
+    float k;
+    int ki;
+};
+__device__ __forceinline__ Draw merge_draw(const Draw &a, const Draw &b)
+{
+    return (b.k > a.k || (b.k == a.k && b.ki < a.ki)) ? b : a;
+}
+
+// Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11): ten rounds of two 32x32->64 multiplies
+// by 0xD2511F53 / 0xCD9E8D57, key bumped by 0x9E3779B9 / 0xBB67AE85 every round.
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                               uint32_t k1)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        c0 = hi1 ^ c1 ^ k0;
+        c1 = lo1;
+        c2 = hi0 ^ c3 ^ k1;
+        c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+// Standard Gumbel variate from one random word: u = (2k + 1) / 2^24 with k its top 23 bits
+// (exact in float32, never 0 or 1), g = -ln(-ln u).
+__device__ __forceinline__ float gumbel_from_word(uint32_t word)
+{
+    const float u = static_cast<float>(2u * (word >> 9) + 1u) * 5.9604644775390625e-8f;   // 2^-24
+    return -logf(-logf(u));
+}
 #endif  // __CUDACC__
 
 struct LmheadParams {
@@ -114,6 +151,13 @@ struct LmheadParams {
     float *part_s;         // sum of exp(z - m)
     float *part_t;         // sum of exp(z - m) * (z - m) * log2(e)
     int32_t *part_i;       // column of the max
+    // sampling (temperature > 0): arg max of z / T + Gumbel noise, kept beside the statistics
+    int32_t sampling;
+    float inv_temperature;
+    uint32_t seed_lo, seed_hi;
+    float *part_k;         // largest perturbed value
+    int32_t *part_ki;      // its column
+    const int32_t *perm;   // compacted row -> caller's row (the random stream is per caller row)
 };
 
 }  // namespace ead

@@ -108,6 +108,9 @@ struct GateParams {
     const RunArgs *args;
     const float *part_m, *part_s, *part_t;
     const int32_t *part_i;
+    int32_t sampling;          // != 0: the token is the sampled candidate, not the arg max
+    const float *part_k;
+    const int32_t *part_ki;
     const int32_t *perm;
     uint8_t *flag;
     int32_t *c;
@@ -140,7 +143,8 @@ __device__ __forceinline__ RowState load_row_state(const GateParams &p, int m, i
     return st;
 }
 
-__device__ __forceinline__ void finish_row(const GateParams &p, const RowState &st, const Partial &acc, int t_step)
+__device__ __forceinline__ void finish_row(const GateParams &p, const RowState &st, const Partial &acc, int t_step,
+                                           const Draw &draw)
 {
     // ---- Eq. 2 in the fused form  H = ln Z - E_p[z] = ln s - t / (s log2 e)   (nats)
     float H = logf(acc.s) - acc.t / (acc.s * kLog2e);
@@ -182,11 +186,23 @@ __device__ __forceinline__ void finish_row(const GateParams &p, const RowState &
     p.flag[b] = static_cast<uint8_t>(model);
     p.usage[used * p.B + b] += 1u;                     // this row is owned by this thread: no atomics
     if (model != used) p.usage[2 * p.B + b] += 1u;
-    if (p.args->tok) p.args->tok[o] = acc.idx;
+    if (p.args->tok) p.args->tok[o] = p.sampling ? draw.ki : acc.idx;
     if (p.args->H) p.args->H[o] = H;
     if (p.args->Hbar) p.args->Hbar[o] = Hbar;
     if (p.args->used) p.args->used[o] = static_cast<uint8_t>(used);
     if (p.args->next) p.args->next[o] = static_cast<uint8_t>(model);
+}
+
+__device__ __forceinline__ Draw warp_merge_draw(Draw d)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Draw q;
+        q.k = __shfl_xor_sync(0xffffffffu, d.k, o);
+        q.ki = __shfl_xor_sync(0xffffffffu, d.ki, o);
+        d = merge_draw(d, q);
+    }
+    return d;
 }
 
 __device__ __forceinline__ Partial warp_merge(Partial acc)
@@ -228,12 +244,15 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const Gate
     //      order, then a butterfly over the lanes (no float atomics: deterministic)
     const size_t base = (static_cast<size_t>(m) * p.B + r) * p.slots_stride;
     Partial acc{kNegSentinel, 0.f, 0.f, 0x7fffffff};
+    Draw draw{-INFINITY, 0x7fffffff};
     for (int s = lane; s < g; s += 32) {
         const Partial q{p.part_m[base + s], p.part_s[base + s], p.part_t[base + s], p.part_i[base + s]};
         acc = merge_partial(acc, q);
+        if (p.sampling) draw = merge_draw(draw, Draw{p.part_k[base + s], p.part_ki[base + s]});
     }
     acc = warp_merge(acc);
-    if (lane == 0) finish_row(p, load_row_state(p, m, r), acc, t_step);
+    if (p.sampling) draw = warp_merge_draw(draw);
+    if (lane == 0) finish_row(p, load_row_state(p, m, r), acc, t_step, draw);
 }
 
 // One block per compacted row: the 4 G partials of the small-batch kernel.  Thread t folds slots t, t + 256, ... in ascending order, then lanes, then warps:
@@ -241,6 +260,7 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const Gate
 __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_wide_kernel(const GateParams p)
 {
     __shared__ Partial wsum[kGateThreads / 32];
+    __shared__ Draw dsum[kGateThreads / 32];
     __shared__ float ring_sh[64];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int i = blockIdx.x;
@@ -270,18 +290,28 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_wide_kernel(const
     if (!live) return;
     const size_t base = (static_cast<size_t>(m) * p.B + r) * p.slots_stride;
     Partial acc{kNegSentinel, 0.f, 0.f, 0x7fffffff};
+    Draw draw{-INFINITY, 0x7fffffff};
     for (int s = threadIdx.x; s < p.n_slots; s += kGateThreads) {
         const Partial q{p.part_m[base + s], p.part_s[base + s], p.part_t[base + s], p.part_i[base + s]};
         acc = merge_partial(acc, q);
+        if (p.sampling) draw = merge_draw(draw, Draw{p.part_k[base + s], p.part_ki[base + s]});
     }
     acc = warp_merge(acc);
-    if (lane == 0) wsum[warp] = acc;
+    if (p.sampling) draw = warp_merge_draw(draw);
+    if (lane == 0) {
+        wsum[warp] = acc;
+        dsum[warp] = draw;
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
         acc = wsum[0];
+        draw = dsum[0];
 #pragma unroll
-        for (int k = 1; k < kGateThreads / 32; ++k) acc = merge_partial(acc, wsum[k]);
-        finish_row(p, st, acc, t_step);
+        for (int k = 1; k < kGateThreads / 32; ++k) {
+            acc = merge_partial(acc, wsum[k]);
+            draw = merge_draw(draw, dsum[k]);
+        }
+        finish_row(p, st, acc, t_step, draw);
     }
 }
 

@@ -125,6 +125,8 @@ __device__ __forceinline__ void rowstat_absorb32(RowStat &st, const float (&v)[3
     st.t = t;
 }
 
+// SAMPLE: also track the arg max of z / T + Gumbel noise (temperature sampling).
+template <bool SAMPLE>
 __global__ void __launch_bounds__(kLmheadThreads, 1)
 ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
                   const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
@@ -277,6 +279,12 @@ ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
             const bool warp_has_rows = quad * 32 < rows_valid;
             RowStat st;
             rowstat_reset(st);
+            // sampling: this thread's sequence draws from its own stream (caller's row, step)
+            Draw dr{-INFINITY, 0x7fffffff};
+            const bool row_live = sp.rb * kTileM + row_in_block < n_rows[m];
+            const bool sampling = SAMPLE && row_live;
+            const uint32_t rng_row = sampling ? static_cast<uint32_t>(p.perm[m * p.B + sp.rb * kTileM + row_in_block]) : 0u;
+            const uint32_t rng_step = static_cast<uint32_t>(p.ctl->cur_t);
             for (int col0 = sp.col_begin; col0 < sp.col_end && ok; col0 += kTileN, ++tc) {
                 const int ncols = min(kTileN, sp.col_end - col0);
                 const uint32_t buf = tc & 1u;
@@ -297,6 +305,23 @@ ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
                             for (int j = 0; j < 32; ++j) v[j] = (cb + j < col_limit) ? v[j] : kNegSentinel;
                         }
                         rowstat_absorb32(st, v, cb);
+                        if (SAMPLE && sampling) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {        // cb is a multiple of 16
+                                const uint4 w = philox4x32_10(static_cast<uint32_t>(cb + j) >> 2, rng_step, rng_row, 0u,
+                                                              p.seed_lo, p.seed_hi);
+                                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    // masked columns hold the sentinel: their value can never win
+                                    const float key = fmaf(v[j + q], p.inv_temperature, gumbel_from_word(ww[q]));
+                                    if (key > dr.k) {
+                                        dr.k = key;
+                                        dr.ki = cb + j + q;
+                                    }
+                                }
+                            }
+                        }
                         __syncwarp();
                     }
                 }
@@ -311,6 +336,10 @@ ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
                 p.part_s[o] = st.s;
                 p.part_t[o] = st.t;
                 p.part_i[o] = st.idx;
+                if (SAMPLE) {
+                    p.part_k[o] = dr.k;
+                    p.part_ki[o] = dr.ki;
+                }
             }
         }
     }

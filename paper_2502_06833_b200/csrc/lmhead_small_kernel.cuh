@@ -38,7 +38,7 @@ constexpr int kSmallWBytes = kSmallTileRows * 64 * 2;  // one 64-wide box of W r
 constexpr int kSmallTmemCols = 32;                     // 2 accumulators x 16 columns
 __host__ __device__ constexpr int small_stage_bytes(int h_rows) { return 2 * h_rows * 128 + 2 * kSmallWBytes; }
 
-template <int NB>
+template <int NB, bool SAMPLE>
 __global__ void __launch_bounds__(kLmheadThreads, 1)
 ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
                         const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
@@ -197,6 +197,17 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                 stt[j] = 0.f;
                 sidx[j] = 0x7fffffff;
             }
+            // sampling: largest perturbed value per sequence; the random stream is per caller's row
+            float dk[NB];
+            int dki[NB];
+            uint32_t rng_row[NB];
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                dk[j] = -INFINITY;
+                dki[j] = 0x7fffffff;
+                rng_row[j] = (SAMPLE && j < n_rows[m]) ? static_cast<uint32_t>(p.perm[m * p.B + j]) : 0u;
+            }
+            const uint32_t rng_step = static_cast<uint32_t>(p.ctl->cur_t);
             for (int row0 = row_begin; row0 < row_end && ok; row0 += kSmallTileRows, ++tc) {
                 const int nrows = min(kSmallTileRows, row_end - row0);
                 const uint32_t buf = tc & 1u;
@@ -226,6 +237,19 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                         sidx[j] = (z > mo) ? row : sidx[j];
                         sm[j] = mn;
                     }
+                    if (SAMPLE) {
+#pragma unroll
+                        for (int j = 0; j < NB; ++j) {
+                            const uint4 w = philox4x32_10(static_cast<uint32_t>(row) >> 2, rng_step, rng_row[j], 0u,
+                                                          p.seed_lo, p.seed_hi);
+                            const uint32_t word = (row & 3) == 0 ? w.x : (row & 3) == 1 ? w.y : (row & 3) == 2 ? w.z : w.w;
+                            const float key = fmaf(v[j], p.inv_temperature, gumbel_from_word(word));
+                            if (key > dk[j]) {            // rows ascend within a thread: lowest row wins ties
+                                dk[j] = key;
+                                dki[j] = row;
+                            }
+                        }
+                    }
                 }
                 __syncwarp();
             }
@@ -250,6 +274,22 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                     p.part_s[o] = acc.s;
                     p.part_t[o] = acc.t;
                     p.part_i[o] = acc.idx;
+                }
+                if (SAMPLE) {
+                    Draw d{dk[j], dki[j]};
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        Draw q;
+                        q.k = __shfl_xor_sync(0xffffffffu, d.k, o);
+                        q.ki = __shfl_xor_sync(0xffffffffu, d.ki, o);
+                        d = merge_draw(d, q);
+                    }
+                    if (lane == 0 && j < n_rows[m]) {
+                        const size_t o = (static_cast<size_t>(m) * p.B + j) * p.slots_stride +
+                                         cta * kSmallSlotsPerCta + quad;
+                        p.part_k[o] = d.k;
+                        p.part_ki[o] = d.ki;
+                    }
                 }
             }
         }

@@ -17,7 +17,7 @@ def to_dev_bf16(bits: np.ndarray):
 class GpuGate:
     """Owns the device copies of one workload and a library context."""
 
-    def __init__(self, cfg, W_small_bits, W_large_bits, stream=None):
+    def __init__(self, cfg, W_small_bits, W_large_bits, stream=None, temperature=0.0, seed=0):
         import torch
         from paper_2502_06833_b200 import binding as E
         self.E, self.torch, self.cfg = E, torch, cfg
@@ -28,7 +28,7 @@ class GpuGate:
                                 d_min=cfg.d_min, tau=cfg.tau, unit=cfg.unit,
                                 start_model=cfg.start_model, W_small=self.W_small,
                                 W_large=self.W_large, device=torch.cuda.current_device(),
-                                stream=self.stream.cuda_stream)
+                                stream=self.stream.cuda_stream, temperature=temperature, seed=seed)
 
     def close(self):
         if self.ctx:

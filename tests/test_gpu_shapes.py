@@ -220,3 +220,28 @@ def test_usage_counters_follow_the_trace_and_survive_a_checkpoint():
                        switches=sum(w[2] for w in want))
     assert tot["tokens_small"] + tot["tokens_large"] == cfg.B * cfg.T
     assert ratio == pytest.approx(O.parameter_ratio(ora["used"].mean(), 1.0, 3.0), rel=1e-12)
+
+
+@pytest.mark.parametrize("B,V,Hs,Hl,temp", [(3, 1000, 64, 128, 1.0), (1, 4100, 256, 512, 0.7),
+                                            (12, 2500, 128, 64, 1.5), (40, 3000, 64, 128, 1.0),
+                                            (130, 1700, 64, 64, 0.8)])
+def test_temperature_sampling_matches_the_oracle_draws(B, V, Hs, Hl, temp):
+    """Algorithm 1's sampling lines: same Philox stream and Gumbel-max rule on both sides, so
+    the drawn tokens must be identical (up to logged near-ties of the perturbed values);
+    entropies and switches are those of the greedy run (entropy is taken before temperature)."""
+    cfg = _cfg(B=B, V=V, H_small=Hs, H_large=Hl, tau=_mid_tau(V), T=16)
+    wl = synth.Workload(cfg)
+    seed = 0x1234567890ABCDEF
+    ora = O.run(wl.W_small, wl.W_large, wl.h_small, wl.h_large, w=cfg.w, d_min=cfg.d_min,
+                tau=float(np.float32(cfg.tau)), temperature=temp, seed=seed)
+    greedy = _oracle(cfg, wl)
+    with GpuGate(cfg, wl.W_small, wl.W_large, temperature=temp, seed=seed) as g:
+        out = g.run(wl.h_small, wl.h_large, "run")
+        g.E.ead_reset(g.ctx)
+        again = g.run(wl.h_small, wl.h_large, "step")
+    log = compare(out, ora, cfg.tau)
+    assert len(log["token_near_ties"]) <= 2
+    assert np.array_equal(out["tok"], again["tok"])                # same stream after a reset
+    assert (ora["tok"] != greedy["tok"]).mean() > 0.2              # the draws are not the arg max
+    assert np.array_equal(out["used"], greedy["used"])
+    assert out["tok"].min() >= 0 and out["tok"].max() < V
