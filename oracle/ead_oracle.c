@@ -242,6 +242,8 @@ void oracle_gate_trace(const double *H, int64_t T, int32_t w, int32_t d_min, dou
 }
 
 /*
+ * A sequence whose token equals eos_token (>= 0) is done: that step is complete, later
+ * steps of the row report token -1, NaN entropies and the unchanged model.
  * Algorithm 1 (greedy for temperature 0, sampled otherwise) for the rows listed in `rows` (n_rows of
  * them, indices into [0, B)) and T tokens.  Inputs are bf16 bit patterns:
  * W_small [V, H_small], W_large [V, H_large], h_small [T, B, H_small],
@@ -257,7 +259,7 @@ void oracle_run(int64_t B, int64_t T, int64_t V, int64_t H_small, int64_t H_larg
                 const uint16_t *h_small, const uint16_t *h_large,
                 const int64_t *rows, int64_t n_rows,
                 int32_t *tok, double *H, double *Hbar, uint8_t *used, uint8_t *next,
-                double *gap, int32_t *c_after, double temperature, uint64_t seed)
+                double *gap, int32_t *c_after, double temperature, uint64_t seed, int32_t eos_token)
 {
     double *z = (double *)malloc((size_t)V * sizeof(double));
     double *hist = (double *)malloc((size_t)(T > 0 ? T : 1) * sizeof(double));
@@ -266,9 +268,19 @@ void oracle_run(int64_t B, int64_t T, int64_t V, int64_t H_small, int64_t H_larg
         int64_t n = 0;                  /* W <- []      */
         int32_t c = 0;                  /* c <- 0       */
         int32_t model = start_model;    /* M_t <- M_S   */
+        int done = 0;                   /* "while not done": set by the end-of-sequence token */
         for (int64_t t = 0; t < T; ++t) {
             int64_t o = t * n_rows + k;
             if (used) used[o] = (uint8_t)model;
+            if (done) {                 /* the loop has ended for this sequence: nothing is computed */
+                if (tok) tok[o] = -1;
+                if (H) H[o] = NAN;
+                if (Hbar) Hbar[o] = NAN;
+                if (next) next[o] = (uint8_t)model;
+                if (gap) gap[o] = NAN;
+                if (c_after) c_after[o] = c;
+                continue;
+            }
             if (model == 0)
                 oracle_logits(W_small, V, H_small, h_small + (t * B + b) * H_small, z);
             else
@@ -286,6 +298,7 @@ void oracle_run(int64_t B, int64_t T, int64_t V, int64_t H_small, int64_t H_larg
             if (next) next[o] = (uint8_t)model;
             if (gap) gap[o] = g;
             if (c_after) c_after[o] = c;
+            if (eos_token >= 0 && tk == eos_token) done = 1;
         }
     }
     free(hist);

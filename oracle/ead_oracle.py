@@ -61,7 +61,7 @@ def lib():
                                  + [C.POINTER(C.c_int32), C.POINTER(C.c_double),
                                     C.POINTER(C.c_double), C.POINTER(C.c_uint8),
                                     C.POINTER(C.c_uint8), C.POINTER(C.c_double),
-                                    C.POINTER(C.c_int32), C.c_double, C.c_uint64])
+                                    C.POINTER(C.c_int32), C.c_double, C.c_uint64, C.c_int32])
         L.oracle_philox4x32.restype = None
         L.oracle_philox4x32.argtypes = [C.POINTER(C.c_uint32)] * 3
         L.oracle_uniform.restype = C.c_double
@@ -177,7 +177,7 @@ def sample(z, temperature: float, seed: int, row: int, step: int):
 
 def run(W_small, W_large, h_small, h_large, *, w: int, d_min: int, tau: float, unit: int = 0,
         start_model: int = 0, rows=None, T: int | None = None, temperature: float = 0.0,
-        seed: int = 0):
+        seed: int = 0, eos_token: int = -1):
     """Algorithm 1 (greedy) on bf16 bit-pattern inputs.
 
     ``h_small``/``h_large`` are ``[T, B, H]`` uint16; ``rows`` selects which of
@@ -209,7 +209,7 @@ def run(W_small, W_large, h_small, h_large, *, w: int, d_min: int, tau: float, u
                      _p(out["tok"], C.c_int32), _p(out["H"], C.c_double),
                      _p(out["Hbar"], C.c_double), _p(out["used"], C.c_uint8),
                      _p(out["next"], C.c_uint8), _p(out["gap"], C.c_double),
-                     _p(out["c_after"], C.c_int32), float(temperature), int(seed))
+                     _p(out["c_after"], C.c_int32), float(temperature), int(seed), int(eos_token))
     return out
 
 

@@ -423,3 +423,24 @@ def test_run_with_temperature_keeps_entropy_and_switches_of_the_greedy_run():
         for bb in range(B):
             z = O.logits(Ws, hs[t, bb]) if b["used"][t, bb] == 0 else O.logits(Wl, hl[t, bb])
             assert b["tok"][t, bb] == O.sample(z, 1.0, 5, bb, t)[0]
+
+
+# ---------------------------------------------------------------- "while not done"
+def test_end_of_sequence_token_stops_a_row_and_only_that_row():
+    r, Ws, Wl, hs, hl = _tiny_inputs()
+    full = O.run(Ws, Wl, hs, hl, w=3, d_min=2, tau=4.6)
+    T, B = r.shape
+    eos = int(full["tok"][6, 1])                      # row 1 emits this token at step 6
+    first = [next((t for t in range(T) if full["tok"][t, b] == eos), None) for b in range(B)]
+    assert first[1] is not None and first[1] <= 6
+    out = O.run(Ws, Wl, hs, hl, w=3, d_min=2, tau=4.6, eos_token=eos)
+    for b in range(B):
+        stop = T if first[b] is None else first[b] + 1            # the step that emits it is complete
+        for k in ("tok", "H", "Hbar", "used", "next", "c_after"):
+            assert np.array_equal(out[k][:stop, b], full[k][:stop, b]), (k, b)
+        assert np.all(out["tok"][stop:, b] == -1)
+        assert np.all(np.isnan(out["H"][stop:, b])) and np.all(np.isnan(out["Hbar"][stop:, b]))
+        if stop < T:
+            assert np.all(out["used"][stop:, b] == full["next"][stop - 1, b])
+            assert np.all(out["next"][stop:, b] == full["next"][stop - 1, b])
+            assert np.all(out["c_after"][stop:, b] == full["c_after"][stop - 1, b])
