@@ -71,6 +71,7 @@ typedef struct ead_config {
     void   *stream;      /* cudaStream_t to enqueue on (borrowed); NULL = legacy default      */
     float   temperature; /* T of Algorithm 1's sampling lines; 0 = greedy (arg max)           */
     uint64_t seed;       /* seed of the sampling random stream (used when temperature > 0)    */
+    int32_t eos_token;   /* token that ends a sequence ("while not done"); < 0 = none         */
 } ead_config;
 
 /*
@@ -161,6 +162,18 @@ int ead_status(ead_ctx *ctx, uint32_t *status_word);
 size_t ead_state_size(const ead_ctx *ctx);
 int ead_get_state(ead_ctx *ctx, void *host_blob, size_t size);
 int ead_set_state(ead_ctx *ctx, const void *host_blob, size_t size);
+
+/*
+ * Done mask ("while not done" of Algorithm 1).  A sequence becomes done when it produces
+ * cfg.eos_token, or when the caller marks it here.  From the next step on a done row takes no
+ * part: no logits are computed for it, its outputs are token -1, NaN entropies and its
+ * unchanged model in model_used / next_model, and its window, counters and model stay frozen.
+ * ead_reset clears the mask.  Both calls wait for the stream.
+ *   done  host, uint8 [B], each 0 or 1
+ * Errors: EAD_EINVALID_ARG, EAD_ECUDA.
+ */
+int ead_set_done(ead_ctx *ctx, const uint8_t *done);
+int ead_get_done(ead_ctx *ctx, uint8_t *done);
 
 /*
  * Usage accounting since the last ead_reset (the paper's "large model usage" column and the

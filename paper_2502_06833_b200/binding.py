@@ -29,14 +29,14 @@ EAD_STATUS_BAD_COUNT = 0x4
 SYMBOLS = ["ead_create", "ead_step", "ead_run", "ead_run_host", "ead_run_timed", "ead_reset", "ead_status",
            "ead_state_size", "ead_get_state", "ead_set_state", "ead_kernel_launches",
            "ead_launch_info", "ead_destroy", "ead_strerror", "ead_head_entropy_static",
-           "ead_plan_split", "ead_usage", "ead_parameter_ratio"]
+           "ead_plan_split", "ead_usage", "ead_parameter_ratio", "ead_set_done", "ead_get_done"]
 
 
 class EadConfig(C.Structure):
     _fields_ = [("B", C.c_int32), ("V", C.c_int32), ("H_small", C.c_int32), ("H_large", C.c_int32),
                 ("w", C.c_int32), ("d_min", C.c_int32), ("tau", C.c_float), ("unit", C.c_int32),
                 ("start_model", C.c_int32), ("device", C.c_int32), ("stream", C.c_void_p),
-                ("temperature", C.c_float), ("seed", C.c_uint64)]
+                ("temperature", C.c_float), ("seed", C.c_uint64), ("eos_token", C.c_int32)]
 
 
 class EadError(RuntimeError):
@@ -87,6 +87,10 @@ def lib() -> C.CDLL:
         L.ead_head_entropy_static.restype = C.c_int
         L.ead_head_entropy_static.argtypes = [vp, vp, C.c_int32, C.c_int32, C.c_int32, i32p, f32p, vp,
                                               C.c_int32, vp]
+        L.ead_set_done.restype = C.c_int
+        L.ead_set_done.argtypes = [vp, vp]
+        L.ead_get_done.restype = C.c_int
+        L.ead_get_done.argtypes = [vp, vp]
         L.ead_usage.restype = C.c_int
         L.ead_usage.argtypes = [vp, C.POINTER(C.c_uint64), vp]
         L.ead_parameter_ratio.restype = C.c_double
@@ -120,11 +124,11 @@ def _ptr(t):
 
 
 def ead_create(*, B, V, H_small, H_large, w, d_min, tau, W_small, W_large, unit=0, start_model=0,
-               device=0, stream=0, temperature=0.0, seed=0):
+               device=0, stream=0, temperature=0.0, seed=0, eos_token=-1):
     """Returns an opaque context handle (int).  ``W_*`` are device bf16 ``[V, H]``; they are
     borrowed, keep them alive until ``ead_destroy``."""
     cfg = EadConfig(B, V, H_small, H_large, w, d_min, float(tau), unit, start_model, device,
-                    C.c_void_p(int(stream)), float(temperature), int(seed))
+                    C.c_void_p(int(stream)), float(temperature), int(seed), int(eos_token))
     out = C.c_void_p()
     _check(lib().ead_create(C.byref(cfg), _ptr(W_small), _ptr(W_large), C.byref(out)), "ead_create")
     return out.value
@@ -203,6 +207,18 @@ def ead_head_entropy_static(W, h, B, V, H, tok=None, H_out=None, status=None, de
     _check(lib().ead_head_entropy_static(_ptr(W), _ptr(h), int(B), int(V), int(H), _ptr(tok),
                                          _ptr(H_out), _ptr(status), int(device),
                                          C.c_void_p(int(stream))), "ead_head_entropy_static")
+
+
+def ead_set_done(ctx, done) -> None:
+    """``done``: uint8 numpy array [B] of 0/1 (host memory)."""
+    _check(lib().ead_set_done(ctx, _ptr(done)), "ead_set_done")
+
+
+def ead_get_done(ctx, B: int):
+    import numpy as np
+    out = np.zeros(B, dtype=np.uint8)
+    _check(lib().ead_get_done(ctx, _ptr(out)), "ead_get_done")
+    return out
 
 
 def ead_usage(ctx, per_row=None) -> dict:

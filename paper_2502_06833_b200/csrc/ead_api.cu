@@ -22,7 +22,7 @@ using namespace ead;
 namespace {
 
 constexpr int kGraphChunk = 32;           // gate steps unrolled in the replayed graph
-constexpr uint32_t kStateMagic = 0x45414432u;   // "EAD2"
+constexpr uint32_t kStateMagic = 0x45414433u;   // "EAD3"
 constexpr size_t kHostStageBytes = 64u << 20;   // per staging buffer of ead_run_host
 
 struct StateHeader {
@@ -77,7 +77,7 @@ struct ead_ctx {
     // device state and scratch (owned)
     StepCtl *ctl = nullptr;
     RunArgs *args = nullptr;
-    uint8_t *flag = nullptr;
+    uint8_t *flag = nullptr, *done = nullptr;
     int32_t *c = nullptr, *nfill = nullptr, *perm = nullptr, *part_i = nullptr, *part_ki = nullptr;
     float *part_k = nullptr;
     uint32_t *usage = nullptr;
@@ -137,7 +137,7 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     cudaError_t e = cudaSuccess;
     if (ev) cudaEventRecord(ev[0], s);
     e = launch(ead_compact_kernel, dim3(cgrid), dim3(kCompactThreads), static_cast<size_t>(c.B) * sizeof(int32_t), s, pdl,
-               x->ctl, x->args, x->flag, c.B, c.H_small, c.H_large, x->hc[0], x->hc[1], x->perm);
+               x->ctl, x->args, x->flag, x->done, c.B, c.H_small, c.H_large, x->hc[0], x->hc[1], x->perm);
     if (e != cudaSuccess) return EAD_ECUDA;
     if (ev) cudaEventRecord(ev[1], s);
 
@@ -211,6 +211,8 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     gp.nfill = x->nfill;
     gp.ring = x->ring;
     gp.usage = x->usage;
+    gp.done = x->done;
+    gp.eos_token = c.eos_token;
     const int rows_per_block = kGateThreads / 32;
     if (x->small_cols)
         e = launch(ead_merge_gate_wide_kernel, dim3(c.B), dim3(kGateThreads), 0, s, pdl, gp);
@@ -364,7 +366,7 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     *out = nullptr;
     if (cfg->B < 1 || cfg->B > 4096 || cfg->V < 1 || cfg->H_small < 8 || cfg->H_large < 8 || cfg->w < 1 ||
         cfg->w > 64 || (cfg->unit != 0 && cfg->unit != 1) || (cfg->start_model != 0 && cfg->start_model != 1) ||
-        !(cfg->temperature >= 0.f) || !(cfg->temperature < 3.0e38f))
+        !(cfg->temperature >= 0.f) || !(cfg->temperature < 3.0e38f) || cfg->eos_token >= cfg->V)
         return EAD_EINVALID_ARG;
     if (cfg->H_small % 8 || cfg->H_large % 8 || !aligned16(W_small) || !aligned16(W_large)) return EAD_EALIGNMENT;
 
@@ -418,7 +420,7 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     if (x->stages < 2) return fail(EAD_ECUDA);
     if (cudaStreamCreateWithFlags(&x->cap_stream, cudaStreamNonBlocking) != cudaSuccess) return fail(EAD_ECUDA);
     if (cudaMalloc(&x->ctl, sizeof(StepCtl)) != cudaSuccess || cudaMalloc(&x->args, sizeof(RunArgs)) != cudaSuccess ||
-        cudaMalloc(&x->flag, B) != cudaSuccess || cudaMalloc(&x->c, 4ull * B) != cudaSuccess ||
+        cudaMalloc(&x->flag, B) != cudaSuccess || cudaMalloc(&x->done, B) != cudaSuccess || cudaMalloc(&x->c, 4ull * B) != cudaSuccess ||
         cudaMalloc(&x->nfill, 4ull * B) != cudaSuccess || cudaMalloc(&x->perm, 8ull * B) != cudaSuccess ||
         cudaMalloc(&x->ring, 4ull * B * cfg->w) != cudaSuccess ||
         cudaMalloc(&x->usage, 12ull * B) != cudaSuccess ||
@@ -494,7 +496,7 @@ int ead_reset(ead_ctx *x)
     const ead_config &c = x->cfg;
     const int threads = 256;
     ead_reset_kernel<<<(c.B + threads - 1) / threads, threads, 0, x->stream>>>(x->ctl, x->flag, x->c, x->nfill,
-                                                                              x->ring, x->usage, c.B, c.w,
+                                                                              x->ring, x->usage, x->done, c.B, c.w,
                                                                               c.start_model);
     x->launches += 1;
     return cudaGetLastError() == cudaSuccess ? EAD_OK : EAD_ECUDA;
@@ -616,7 +618,7 @@ size_t ead_state_size(const ead_ctx *x)
 {
     if (!x) return 0;
     const size_t B = x->cfg.B;
-    return sizeof(StateHeader) + B /*flag*/ + ((4 - B % 4) % 4) + 4 * B /*c*/ + 4 * B /*nfill*/ + 12 * B /*usage*/ +
+    return sizeof(StateHeader) + 2 * (B + ((4 - B % 4) % 4)) /*flag, done*/ + 4 * B /*c*/ + 4 * B /*nfill*/ + 12 * B /*usage*/ +
            4 * B * x->cfg.w;
 }
 
@@ -633,6 +635,9 @@ int ead_get_state(ead_ctx *x, void *blob, size_t size)
     memcpy(p, &hd, sizeof hd);
     p += sizeof hd;
     EAD_CUDA(cudaMemcpy(p, x->flag, B, cudaMemcpyDeviceToHost));
+    memset(p + B, 0, pad);
+    p += B + pad;
+    EAD_CUDA(cudaMemcpy(p, x->done, B, cudaMemcpyDeviceToHost));
     memset(p + B, 0, pad);
     p += B + pad;
     EAD_CUDA(cudaMemcpy(p, x->c, 4 * B, cudaMemcpyDeviceToHost));
@@ -657,9 +662,11 @@ int ead_set_state(ead_ctx *x, const void *blob, size_t size)
     const size_t B = x->cfg.B, pad = (4 - B % 4) % 4;
     p += sizeof hd;
     for (size_t i = 0; i < B; ++i)
-        if (p[i] > 1) return EAD_ESTATE;
+        if (p[i] > 1 || p[B + pad + i] > 1) return EAD_ESTATE;
     EAD_CUDA(cudaMemcpy(&x->ctl->step, &hd.step, 4, cudaMemcpyHostToDevice));
     EAD_CUDA(cudaMemcpy(x->flag, p, B, cudaMemcpyHostToDevice));
+    p += B + pad;
+    EAD_CUDA(cudaMemcpy(x->done, p, B, cudaMemcpyHostToDevice));
     p += B + pad;
     EAD_CUDA(cudaMemcpy(x->c, p, 4 * B, cudaMemcpyHostToDevice));
     p += 4 * B;
@@ -692,6 +699,24 @@ double ead_parameter_ratio(uint64_t tokens_small, uint64_t tokens_large, double 
     const double total = static_cast<double>(tokens_small) + static_cast<double>(tokens_large);
     const double alpha = static_cast<double>(tokens_small) / total, beta = static_cast<double>(tokens_large) / total;
     return (alpha * P_small + beta * P_large) / P_large;
+}
+
+int ead_set_done(ead_ctx *x, const uint8_t *done)
+{
+    if (!x || !done) return EAD_EINVALID_ARG;
+    for (int b = 0; b < x->cfg.B; ++b)
+        if (done[b] > 1) return EAD_EINVALID_ARG;
+    EAD_CUDA(cudaStreamSynchronize(x->stream));
+    EAD_CUDA(cudaMemcpy(x->done, done, x->cfg.B, cudaMemcpyHostToDevice));
+    return EAD_OK;
+}
+
+int ead_get_done(ead_ctx *x, uint8_t *done)
+{
+    if (!x || !done) return EAD_EINVALID_ARG;
+    EAD_CUDA(cudaStreamSynchronize(x->stream));
+    EAD_CUDA(cudaMemcpy(done, x->done, x->cfg.B, cudaMemcpyDeviceToHost));
+    return EAD_OK;
 }
 
 int64_t ead_kernel_launches(const ead_ctx *x) { return x ? x->launches : 0; }
@@ -730,7 +755,7 @@ void ead_destroy(ead_ctx *x)
     if (x->g_chunk) cudaGraphExecDestroy(x->g_chunk);
     if (x->cap_stream) cudaStreamDestroy(x->cap_stream);
     void *bufs[] = {x->ctl, x->args, x->flag, x->c, x->nfill, x->perm, x->ring, x->hc[0], x->hc[1],
-                    x->part_m, x->part_s, x->part_t, x->part_i, x->usage, x->part_k, x->part_ki};
+                    x->part_m, x->part_s, x->part_t, x->part_i, x->usage, x->part_k, x->part_ki, x->done};
     for (void *b : bufs)
         if (b) cudaFree(b);
     cudaGetLastError();

@@ -28,7 +28,8 @@ struct StepCtl {
     int32_t cur_t;      // copy of `step` taken by the compaction kernel for this step
     int32_t n[2];       // rows served by the small / large head in this step
     uint32_t status;    // sticky EAD_STATUS_* bits
-    int32_t pad[3];
+    int32_t n_done;     // rows whose sequence has ended (served by neither head)
+    int32_t pad[2];
 };
 
 // Caller buffers of the current ead_step / ead_run call (device resident so that a

@@ -23,32 +23,35 @@ __global__ void ead_set_args_kernel(RunArgs *dst, RunArgs a, const StepCtl *ctl)
 }
 
 __global__ void ead_reset_kernel(StepCtl *ctl, uint8_t *flag, int32_t *c, int32_t *nfill, float *ring,
-                                 uint32_t *usage, int B, int w, int start_model)
+                                 uint32_t *usage, uint8_t *done, int B, int w, int start_model)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i == 0) {
         ctl->step = 0;
         ctl->cur_t = 0;
         ctl->n[0] = ctl->n[1] = 0;
+        ctl->n_done = 0;
         ctl->status = 0;
     }
     if (i < B) {
         flag[i] = static_cast<uint8_t>(start_model);
         c[i] = 0;
         nfill[i] = 0;
+        done[i] = 0;
         usage[i] = usage[B + i] = usage[2 * B + i] = 0u;
     }
     for (int k = i; k < B * w; k += gridDim.x * blockDim.x) ring[k] = 0.f;
 }
 
-// Stable partition of the rows by model flag.  Every CTA recomputes the (tiny) scan
-// over the B flags and then copies the rows b = blockIdx.x, blockIdx.x + gridDim.x, ...
-// perm[m * B + r] = original row of compacted row r of head m.
+// Stable partition of the rows by model flag; rows whose sequence has ended ("done") go to
+// neither head and get their outputs here (token -1, NaN entropies, model unchanged).  Every
+// CTA recomputes the (tiny) scan over the B flags and then copies the rows b = blockIdx.x,
+// blockIdx.x + gridDim.x, ...   perm[m * B + r] = original row of compacted row r of head m.
 __global__ void __launch_bounds__(kCompactThreads)
-ead_compact_kernel(StepCtl *ctl, const RunArgs *args, const uint8_t *flag, int B, int Hs, int Hl,
-                   uint16_t *hc_s, uint16_t *hc_l, int32_t *perm)
+ead_compact_kernel(StepCtl *ctl, const RunArgs *args, const uint8_t *flag, const uint8_t *done, int B, int Hs,
+                   int Hl, uint16_t *hc_s, uint16_t *hc_l, int32_t *perm)
 {
-    extern __shared__ int32_t pos_sh[];          // [B]: position | model << 30
+    extern __shared__ uint32_t pos_sh[];         // [B]: position | class << 30 (0 small, 1 large, 2 done)
     __shared__ int32_t warp_tot[kCompactThreads / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     griddep_launch_dependents();                 // the LM-head kernel may set itself up meanwhile
@@ -58,9 +61,9 @@ ead_compact_kernel(StepCtl *ctl, const RunArgs *args, const uint8_t *flag, int B
 
     const int per = (B + kCompactThreads - 1) / kCompactThreads;
     const int b0 = min(B, tid * per), b1 = min(B, b0 + per);
-    int cnt = 0;
-    for (int b = b0; b < b1; ++b) cnt += flag[b] ? 1 : 0;
-    int incl = cnt;                               // inclusive scan of the large-model counts
+    int cnt = 0;                                  // large rows in the low half, done rows in the high half
+    for (int b = b0; b < b1; ++b) cnt += done[b] ? 0x10000 : (flag[b] ? 1 : 0);
+    int incl = cnt;                               // inclusive scan of both counts at once (B <= 4096)
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const int y = __shfl_up_sync(0xffffffffu, incl, o);
@@ -68,31 +71,50 @@ ead_compact_kernel(StepCtl *ctl, const RunArgs *args, const uint8_t *flag, int B
     }
     if (lane == 31) warp_tot[warp] = incl;
     __syncthreads();
-    int before = 0, total_large = 0;
+    int before = 0, total = 0;
 #pragma unroll
     for (int k = 0; k < kCompactThreads / 32; ++k) {
         const int v = warp_tot[k];
         if (k < warp) before += v;
-        total_large += v;
+        total += v;
     }
-    int pos_l = before + incl - cnt;              // large rows before b0
-    int pos_s = b0 - pos_l;                       // small rows before b0
+    const int excl = before + incl - cnt;
+    int pos_l = excl & 0xffff;                    // large rows before b0
+    int pos_s = b0 - pos_l - (excl >> 16);        // small rows before b0
     for (int b = b0; b < b1; ++b) {
+        if (done[b]) {
+            pos_sh[b] = 2u << 30;
+            continue;
+        }
         const int f = flag[b] ? 1 : 0;
         const int pos = f ? pos_l++ : pos_s++;
-        pos_sh[b] = pos | (f << 30);
+        pos_sh[b] = static_cast<uint32_t>(pos) | (static_cast<uint32_t>(f) << 30);
         if (blockIdx.x == 0) perm[f * B + pos] = b;
     }
     if (blockIdx.x == 0 && tid == 0) {
-        ctl->n[0] = B - total_large;
+        const int total_large = total & 0xffff, total_done = total >> 16;
+        ctl->n[0] = B - total_large - total_done;
         ctl->n[1] = total_large;
+        ctl->n_done = total_done;
         ctl->cur_t = step;
     }
     __syncthreads();
 
     for (int b = blockIdx.x; b < B; b += gridDim.x) {
-        const int e = pos_sh[b];
-        const int f = e >> 30, pos = e & 0x3fffffff;
+        const uint32_t e = pos_sh[b];
+        const int f = static_cast<int>(e >> 30), pos = static_cast<int>(e & 0x3fffffffu);
+        if (f == 2) {                             // ended sequence: nothing is computed for it
+            if (tid == 0) {
+                const size_t o = static_cast<size_t>(idx) * B + b;
+                const float nan = __int_as_float(0x7fc00000);
+                if (args->tok) args->tok[o] = -1;
+                if (args->H) args->H[o] = nan;
+                if (args->Hbar) args->Hbar[o] = nan;
+                if (args->used) args->used[o] = flag[b];
+                if (args->next) args->next[o] = flag[b];
+            }
+            continue;
+        }
         const int H = f ? Hl : Hs;
         const uint4 *src = reinterpret_cast<const uint4 *>(args->h[f] + (static_cast<size_t>(idx) * B + b) * H);
         uint4 *dst = reinterpret_cast<uint4 *>((f ? hc_l : hc_s) + static_cast<size_t>(pos) * H);
@@ -117,6 +139,8 @@ struct GateParams {
     int32_t *nfill;
     float *ring;
     uint32_t *usage;           // [3][B]: tokens by the small model, by the large model, switches
+    uint8_t *done;             // [B]: the sequence has produced the end-of-sequence token
+    int32_t eos_token;         // < 0: none
 };
 
 // Everything after the merge for one compacted row (executed by one thread): Eq. 2 in the
@@ -186,7 +210,9 @@ __device__ __forceinline__ void finish_row(const GateParams &p, const RowState &
     p.flag[b] = static_cast<uint8_t>(model);
     p.usage[used * p.B + b] += 1u;                     // this row is owned by this thread: no atomics
     if (model != used) p.usage[2 * p.B + b] += 1u;
-    if (p.args->tok) p.args->tok[o] = p.sampling ? draw.ki : acc.idx;
+    const int token = p.sampling ? draw.ki : acc.idx;
+    if (p.eos_token >= 0 && token == p.eos_token) p.done[b] = 1;    // "while not done" ends for this row
+    if (p.args->tok) p.args->tok[o] = token;
     if (p.args->H) p.args->H[o] = H;
     if (p.args->Hbar) p.args->Hbar[o] = Hbar;
     if (p.args->used) p.args->used[o] = static_cast<uint8_t>(used);
@@ -228,11 +254,12 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const Gate
     griddep_wait();                              // partials of the LM-head kernel
     const int n0 = p.ctl->n[0], n1 = p.ctl->n[1];
     const int t_step = p.ctl->cur_t;
+    const int nd = p.ctl->n_done;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
-        if (n0 + n1 != p.B) atomicOr(&p.ctl->status, kStatusBadCount);
+        if (n0 + n1 + nd != p.B) atomicOr(&p.ctl->status, kStatusBadCount);
         p.ctl->step = t_step + 1;                 // nobody in this kernel reads `step`
     }
-    if (i >= p.B || n0 + n1 != p.B) return;
+    if (i >= n0 + n1 || n0 + n1 + nd != p.B) return;
     const int m = i < n0 ? 0 : 1;
     const int r = m ? i - n0 : i;
     const int n_m = m ? n1 : n0;
@@ -271,7 +298,8 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_wide_kernel(const
     // LM-head kernel.  Only the partials need the wait below.
     const int n0 = p.ctl->n[0], n1 = p.ctl->n[1];
     const int t_step = p.ctl->cur_t;
-    const bool live = i < p.B && n0 + n1 == p.B;
+    const int nd = p.ctl->n_done;
+    const bool live = i < n0 + n1 && n0 + n1 + nd == p.B;
     const int m = i < n0 ? 0 : 1;
     const int r = m ? i - n0 : i;
     RowState st{};
@@ -284,7 +312,7 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_wide_kernel(const
     __syncthreads();
     griddep_wait();                              // partials of the LM-head kernel
     if (blockIdx.x == 0 && threadIdx.x == 0) {
-        if (n0 + n1 != p.B) atomicOr(&p.ctl->status, kStatusBadCount);
+        if (n0 + n1 + nd != p.B) atomicOr(&p.ctl->status, kStatusBadCount);
         p.ctl->step = t_step + 1;
     }
     if (!live) return;

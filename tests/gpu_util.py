@@ -17,7 +17,8 @@ def to_dev_bf16(bits: np.ndarray):
 class GpuGate:
     """Owns the device copies of one workload and a library context."""
 
-    def __init__(self, cfg, W_small_bits, W_large_bits, stream=None, temperature=0.0, seed=0):
+    def __init__(self, cfg, W_small_bits, W_large_bits, stream=None, temperature=0.0, seed=0,
+                 eos_token=-1):
         import torch
         from paper_2502_06833_b200 import binding as E
         self.E, self.torch, self.cfg = E, torch, cfg
@@ -28,7 +29,8 @@ class GpuGate:
                                 d_min=cfg.d_min, tau=cfg.tau, unit=cfg.unit,
                                 start_model=cfg.start_model, W_small=self.W_small,
                                 W_large=self.W_large, device=torch.cuda.current_device(),
-                                stream=self.stream.cuda_stream, temperature=temperature, seed=seed)
+                                stream=self.stream.cuda_stream, temperature=temperature, seed=seed,
+                                eos_token=eos_token)
 
     def close(self):
         if self.ctx:
@@ -93,6 +95,11 @@ def compare(gpu: dict, ora: dict, tau: float, rows=None, unit: int = 0):
     for k, b in enumerate(rows):
         for t in range(T):
             assert gpu["used"][t, b] == ora["used"][t, k], f"model_used differs at t={t} row={b}"
+            if np.isnan(ora["H"][t, k]):           # ended sequence or non-finite logits: same report
+                assert np.isnan(gpu["H"][t, b]) and np.isnan(gpu["Hbar"][t, b]) and gpu["tok"][t, b] == -1
+                assert gpu["next"][t, b] == ora["next"][t, k]
+                log["cells"] += 1
+                continue
             errH = abs(float(gpu["H"][t, b]) - ora["H"][t, k])
             assert errH <= H_TOL_NATS * scale, f"H differs by {errH} at t={t} row={b}"
             log["max_H_err"] = max(log["max_H_err"], errH)

@@ -245,3 +245,31 @@ def test_temperature_sampling_matches_the_oracle_draws(B, V, Hs, Hl, temp):
     assert (ora["tok"] != greedy["tok"]).mean() > 0.2              # the draws are not the arg max
     assert np.array_equal(out["used"], greedy["used"])
     assert out["tok"].min() >= 0 and out["tok"].max() < V
+
+
+@pytest.mark.parametrize("B,V", [(6, 1200), (150, 900)])
+def test_end_of_sequence_token_and_done_mask(B, V):
+    cfg = _cfg(B=B, V=V, T=24, tau=_mid_tau(V))
+    wl = synth.Workload(cfg)
+    free = _oracle(cfg, wl)
+    toks, counts = np.unique(free["tok"][4:12], return_counts=True)
+    eos = int(toks[np.argmax(counts)])                      # ends at least one row mid-run
+    ora = O.run(wl.W_small, wl.W_large, wl.h_small, wl.h_large, w=cfg.w, d_min=cfg.d_min,
+                tau=float(np.float32(cfg.tau)), eos_token=eos)
+    ended = np.isnan(ora["H"][-1])
+    assert ended.any() and not ended.all()
+    with GpuGate(cfg, wl.W_small, wl.W_large, eos_token=eos) as g:
+        out = g.run(wl.h_small, wl.h_large, "run")
+        assert np.array_equal(g.E.ead_get_done(g.ctx, B).astype(bool), ended)
+        blob = g.E.ead_get_state(g.ctx)
+        # a row marked done by the caller stops as well; reset clears the mask
+        g.E.ead_reset(g.ctx)
+        assert not g.E.ead_get_done(g.ctx, B).any()
+        mask = np.zeros(B, dtype=np.uint8)
+        mask[1] = 1
+        g.E.ead_set_done(g.ctx, mask)
+        one = g.run(wl.h_small[:3], wl.h_large[:3], "run")
+    compare(out, ora, cfg.tau)
+    assert np.all(one["tok"][:, 1] == -1) and np.all(np.isnan(one["H"][:, 1]))
+    assert np.array_equal(one["tok"][:, 0], free["tok"][:3, 0])
+    assert len(blob) > 0
