@@ -72,6 +72,9 @@ typedef struct ead_config {
     float   temperature; /* T of Algorithm 1's sampling lines; 0 = greedy (arg max)           */
     uint64_t seed;       /* seed of the sampling random stream (used when temperature > 0)    */
     int32_t eos_token;   /* token that ends a sequence ("while not done"); < 0 = none         */
+    int32_t V_large;     /* vocabulary of M_L if it differs from V (the paper allows models of
+                            different architectures); 0 = same as V.  Tokens of a step are
+                            indices into the vocabulary of the model that produced them      */
 } ead_config;
 
 /*
@@ -79,7 +82,7 @@ typedef struct ead_config {
  * initialisation (empty window, c = 0, M_t = start_model) plus scratch, and
  * encodes the TMA descriptors of the two heads.
  *   W_small  dev, bf16 [V, H_small], one row per vocabulary entry (borrowed, read only)
- *   W_large  dev, bf16 [V, H_large]
+ *   W_large  dev, bf16 [V_large or V, H_large]
  *   out      host, receives the context
  * Synchronises the device once.  Errors: EAD_EINVALID_ARG, EAD_EALIGNMENT,
  * EAD_EUNSUPPORTED_ARCH, EAD_ECUDA.

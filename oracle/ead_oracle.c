@@ -253,7 +253,7 @@ void oracle_gate_trace(const double *H, int64_t T, int32_t w, int32_t d_min, dou
  *   after the switch test), gap (difference of the two largest logits),
  *   c_after (dwell counter after the step).  Any output pointer may be NULL.
  */
-void oracle_run(int64_t B, int64_t T, int64_t V, int64_t H_small, int64_t H_large,
+void oracle_run(int64_t B, int64_t T, int64_t V, int64_t V_large, int64_t H_small, int64_t H_large,
                 int32_t w, int32_t d_min, double tau, int32_t unit, int32_t start_model,
                 const uint16_t *W_small, const uint16_t *W_large,
                 const uint16_t *h_small, const uint16_t *h_large,
@@ -261,7 +261,7 @@ void oracle_run(int64_t B, int64_t T, int64_t V, int64_t H_small, int64_t H_larg
                 int32_t *tok, double *H, double *Hbar, uint8_t *used, uint8_t *next,
                 double *gap, int32_t *c_after, double temperature, uint64_t seed, int32_t eos_token)
 {
-    double *z = (double *)malloc((size_t)V * sizeof(double));
+    double *z = (double *)malloc((size_t)(V > V_large ? V : V_large) * sizeof(double));
     double *hist = (double *)malloc((size_t)(T > 0 ? T : 1) * sizeof(double));
     for (int64_t k = 0; k < n_rows; ++k) {
         int64_t b = rows[k];
@@ -281,16 +281,18 @@ void oracle_run(int64_t B, int64_t T, int64_t V, int64_t H_small, int64_t H_larg
                 if (c_after) c_after[o] = c;
                 continue;
             }
+            /* the two models may have different vocabularies (V for M_S, V_large for M_L) */
+            int64_t Vm = model == 0 ? V : V_large;
             if (model == 0)
-                oracle_logits(W_small, V, H_small, h_small + (t * B + b) * H_small, z);
+                oracle_logits(W_small, Vm, H_small, h_small + (t * B + b) * H_small, z);
             else
-                oracle_logits(W_large, V, H_large, h_large + (t * B + b) * H_large, z);
-            double Ht = oracle_entropy(z, V, unit, NULL);
+                oracle_logits(W_large, Vm, H_large, h_large + (t * B + b) * H_large, z);
+            double Ht = oracle_entropy(z, Vm, unit, NULL);
             double g;
             /* the entropy above is taken before any temperature scaling; the token is the
                arg max (temperature 0) or a draw from softmax(l / T) */
-            int64_t tk = temperature > 0.0 ? oracle_sample(z, V, temperature, seed, b, t, &g)
-                                           : oracle_greedy(z, V, &g);
+            int64_t tk = temperature > 0.0 ? oracle_sample(z, Vm, temperature, seed, b, t, &g)
+                                           : oracle_greedy(z, Vm, &g);
             double Hb = oracle_gate_step(hist, &n, &c, &model, Ht, w, d_min, tau);
             if (tok) tok[o] = (int32_t)tk;
             if (H) H[o] = Ht;

@@ -54,7 +54,7 @@ def lib():
                                        C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.c_double,
                                        C.c_int32, C.c_int32, C.c_double]
         L.oracle_run.restype = None
-        L.oracle_run.argtypes = ([C.c_int64] * 5 + [C.c_int32, C.c_int32, C.c_double, C.c_int32,
+        L.oracle_run.argtypes = ([C.c_int64] * 6 + [C.c_int32, C.c_int32, C.c_double, C.c_int32,
                                                     C.c_int32]
                                  + [C.POINTER(C.c_uint16)] * 4
                                  + [C.POINTER(C.c_int64), C.c_int64]
@@ -192,7 +192,8 @@ def run(W_small, W_large, h_small, h_large, *, w: int, d_min: int, tau: float, u
     Hl = h_large.shape[2]
     assert h_large.shape[:2] == (Tfull, B)
     V = W_small.shape[0]
-    assert W_small.shape == (V, Hs) and W_large.shape == (V, Hl)
+    Vl = W_large.shape[0]
+    assert W_small.shape == (V, Hs) and W_large.shape == (Vl, Hl)
     T = Tfull if T is None else int(T)
     assert 0 <= T <= Tfull
     rows = np.arange(B, dtype=np.int64) if rows is None else np.ascontiguousarray(rows, np.int64)
@@ -201,7 +202,7 @@ def run(W_small, W_large, h_small, h_large, *, w: int, d_min: int, tau: float, u
                Hbar=np.empty((T, n), np.float64), used=np.empty((T, n), np.uint8),
                next=np.empty((T, n), np.uint8), gap=np.empty((T, n), np.float64),
                c_after=np.empty((T, n), np.int32), rows=rows)
-    lib().oracle_run(B, T, V, Hs, Hl, int(w), int(d_min), float(tau), int(unit),
+    lib().oracle_run(B, T, V, Vl, Hs, Hl, int(w), int(d_min), float(tau), int(unit),
                      int(start_model),
                      _p(W_small, C.c_uint16), _p(W_large, C.c_uint16),
                      _p(h_small, C.c_uint16), _p(h_large, C.c_uint16),

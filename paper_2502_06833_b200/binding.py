@@ -36,7 +36,8 @@ class EadConfig(C.Structure):
     _fields_ = [("B", C.c_int32), ("V", C.c_int32), ("H_small", C.c_int32), ("H_large", C.c_int32),
                 ("w", C.c_int32), ("d_min", C.c_int32), ("tau", C.c_float), ("unit", C.c_int32),
                 ("start_model", C.c_int32), ("device", C.c_int32), ("stream", C.c_void_p),
-                ("temperature", C.c_float), ("seed", C.c_uint64), ("eos_token", C.c_int32)]
+                ("temperature", C.c_float), ("seed", C.c_uint64), ("eos_token", C.c_int32),
+                ("V_large", C.c_int32)]
 
 
 class EadError(RuntimeError):
@@ -124,11 +125,11 @@ def _ptr(t):
 
 
 def ead_create(*, B, V, H_small, H_large, w, d_min, tau, W_small, W_large, unit=0, start_model=0,
-               device=0, stream=0, temperature=0.0, seed=0, eos_token=-1):
+               device=0, stream=0, temperature=0.0, seed=0, eos_token=-1, V_large=0):
     """Returns an opaque context handle (int).  ``W_*`` are device bf16 ``[V, H]``; they are
     borrowed, keep them alive until ``ead_destroy``."""
     cfg = EadConfig(B, V, H_small, H_large, w, d_min, float(tau), unit, start_model, device,
-                    C.c_void_p(int(stream)), float(temperature), int(seed), int(eos_token))
+                    C.c_void_p(int(stream)), float(temperature), int(seed), int(eos_token), int(V_large))
     out = C.c_void_p()
     _check(lib().ead_create(C.byref(cfg), _ptr(W_small), _ptr(W_large), C.byref(out)), "ead_create")
     return out.value

@@ -70,6 +70,7 @@ struct ead_ctx {
     cudaStream_t stream = nullptr;
     cudaStream_t cap_stream = nullptr;     // capture happens on a private stream
     int G = 0, a_rows = 0, stages = 0, slots_stride = 0;
+    int V_large = 0;                       // vocabulary of the large head (cfg.V_large, or cfg.V if that is 0)
     int small_cols = 0;                    // > 0: swapped-operand kernel with this many batch columns
     int small_slots = 0;                   // partial slots per row it writes (one per CTA and epilogue warp)
     size_t smem_bytes = 0;
@@ -142,7 +143,8 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     if (ev) cudaEventRecord(ev[1], s);
 
     LmheadParams lp{};
-    lp.V = c.V;
+    lp.V[0] = c.V;
+    lp.V[1] = x->V_large;
     lp.H[0] = c.H_small;
     lp.H[1] = c.H_large;
     lp.a_rows = x->a_rows;
@@ -366,7 +368,8 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     *out = nullptr;
     if (cfg->B < 1 || cfg->B > 4096 || cfg->V < 1 || cfg->H_small < 8 || cfg->H_large < 8 || cfg->w < 1 ||
         cfg->w > 64 || (cfg->unit != 0 && cfg->unit != 1) || (cfg->start_model != 0 && cfg->start_model != 1) ||
-        !(cfg->temperature >= 0.f) || !(cfg->temperature < 3.0e38f) || cfg->eos_token >= cfg->V)
+        !(cfg->temperature >= 0.f) || !(cfg->temperature < 3.0e38f) || cfg->V_large < 0 ||
+        cfg->eos_token >= std::min(cfg->V, cfg->V_large > 0 ? cfg->V_large : cfg->V))
         return EAD_EINVALID_ARG;
     if (cfg->H_small % 8 || cfg->H_large % 8 || !aligned16(W_small) || !aligned16(W_large)) return EAD_EALIGNMENT;
 
@@ -382,6 +385,7 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     if (!x) return EAD_ECUDA;
     x->cfg = *cfg;
     x->stream = static_cast<cudaStream_t>(cfg->stream);
+    x->V_large = cfg->V_large > 0 ? cfg->V_large : cfg->V;
     x->W[0] = W_small;
     x->W[1] = W_large;
     x->G = std::min(prop.multiProcessorCount, kMaxCtas);
@@ -442,14 +446,15 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     cudaMemsetAsync(x->part_k, 0, 4 * np, x->stream);
     cudaMemsetAsync(x->part_ki, 0, 4 * np, x->stream);
 
-    const uint32_t wbox = static_cast<uint32_t>(
-        std::min(x->small_cols ? kSmallTileRows : kTileN, (cfg->V + kUnit - 1) / kUnit * kUnit));
     const int Hm[2] = {cfg->H_small, cfg->H_large};
+    const int Vm[2] = {cfg->V, x->V_large};
     for (int m = 0; m < 2; ++m) {
+        const uint32_t wbox = static_cast<uint32_t>(
+            std::min(x->small_cols ? kSmallTileRows : kTileN, (Vm[m] + kUnit - 1) / kUnit * kUnit));
         if (!encode_bf16_2d(&x->tmA[m], x->hc[m], Bpad, Hm[m], x->a_rows) ||
-            !encode_bf16_2d(&x->tmW[m], x->W[m], cfg->V, Hm[m], wbox) ||
-            !encode_bf16_2d(&x->tmT[m], x->W[m], cfg->V, Hm[m], kUnit) ||
-            !encode_bf16_2d(&x->tmP[m], x->W[m], cfg->V, Hm[m], kSmallSegRows))
+            !encode_bf16_2d(&x->tmW[m], x->W[m], Vm[m], Hm[m], wbox) ||
+            !encode_bf16_2d(&x->tmT[m], x->W[m], Vm[m], Hm[m], kUnit) ||
+            !encode_bf16_2d(&x->tmP[m], x->W[m], Vm[m], Hm[m], kSmallSegRows))
             return fail(EAD_ECUDA);
     }
     // the attribute belongs to the kernel on this device, not to the context: ask for the
@@ -916,7 +921,8 @@ extern "C" int ead_head_entropy_static(const void *W, const void *h, int32_t B, 
     ead_static_clear_status_kernel<<<1, 1, 0, s>>>(status);
     ead_static_stage_kernel<<<a_rows, 128, 0, s>>>(sc, static_cast<const uint16_t *>(h), B, H, a_rows);
     LmheadParams lp{};
-    lp.V = V;
+    lp.V[0] = V;
+    lp.V[1] = V;
     lp.H[0] = H;
     lp.H[1] = H;
     lp.a_rows = a_rows;

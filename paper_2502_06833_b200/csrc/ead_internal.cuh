@@ -139,7 +139,7 @@ __device__ __forceinline__ float gumbel_from_word(uint32_t word)
 #endif  // __CUDACC__
 
 struct LmheadParams {
-    int32_t V;
+    int32_t V[2];          // vocabulary size of the small / large head
     int32_t H[2];
     int32_t a_rows;        // rows of the hidden-state TMA box (multiple of 8, <= 128)
     int32_t n_cols;        // small-batch kernel: batch columns kept per thread (power of two <= 16)

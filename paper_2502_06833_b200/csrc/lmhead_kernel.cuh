@@ -189,7 +189,7 @@ ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
             uint32_t it = 0;
             bool ok = true;
             for (int m = 0; m < 2 && ok; ++m) {
-                const HeadSplit sp = split_head(cta, G, n_rows[m], p.V);
+                const HeadSplit sp = split_head(cta, G, n_rows[m], p.V[m]);
                 if (!sp.active) continue;
                 const CUtensorMap *tA = m ? &tmA1 : &tmA0;
                 const CUtensorMap *tW = m ? &tmW1 : &tmW0;
@@ -231,7 +231,7 @@ ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
             uint32_t it = 0, tc = 0;
             bool ok = true;
             for (int m = 0; m < 2 && ok; ++m) {
-                const HeadSplit sp = split_head(cta, G, n_rows[m], p.V);
+                const HeadSplit sp = split_head(cta, G, n_rows[m], p.V[m]);
                 if (!sp.active) continue;
                 const int kblocks = (p.H[m] + kBlockK - 1) / kBlockK;
                 for (int col0 = sp.col_begin; col0 < sp.col_end && ok; col0 += kTileN, ++tc) {
@@ -273,7 +273,7 @@ ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
         uint32_t tc = 0;
         bool ok = true;
         for (int m = 0; m < 2 && ok; ++m) {
-            const HeadSplit sp = split_head(cta, G, n_rows[m], p.V);
+            const HeadSplit sp = split_head(cta, G, n_rows[m], p.V[m]);
             if (!sp.active) continue;
             const int rows_valid = min(kTileM, n_rows[m] - sp.rb * kTileM);
             const bool warp_has_rows = quad * 32 < rows_valid;
@@ -294,7 +294,7 @@ ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
                 }
                 tc_fence_after_sync();
                 if (warp_has_rows) {
-                    const int col_limit = min(p.V, col0 + ncols);       // first invalid column
+                    const int col_limit = min(p.V[m], col0 + ncols);       // first invalid column
                     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + buf * kTileN;
                     for (int c = 0; c < ncols; c += 32) {
                         float v[32];

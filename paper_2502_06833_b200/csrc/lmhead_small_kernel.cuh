@@ -88,11 +88,14 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
     // Everything above touched no global memory: it may overlap the kernels before this one.
     griddep_wait();
     griddep_launch_dependents();
-    const int v_pad = (p.V + kSmallSegRows - 1) / kSmallSegRows * kSmallSegRows;
-    const int n_seg = v_pad / kSmallSegRows;
     const int cta = blockIdx.x;
-    const int row_begin = static_cast<int>(static_cast<long long>(n_seg) * cta / G) * kSmallSegRows;
-    const int row_end = static_cast<int>(static_cast<long long>(n_seg) * (cta + 1) / G) * kSmallSegRows;
+    int row_begin_m[2], row_end_m[2];            // this CTA's vocabulary range on each head
+#pragma unroll
+    for (int m = 0; m < 2; ++m) {
+        const long long n_seg = (p.V[m] + kSmallSegRows - 1) / kSmallSegRows;
+        row_begin_m[m] = static_cast<int>(n_seg * cta / G) * kSmallSegRows;
+        row_end_m[m] = static_cast<int>(n_seg * (cta + 1) / G) * kSmallSegRows;
+    }
     const int n_rows[2] = {p.ctl->n[0], p.ctl->n[1]};
 
     if (warp == 0) {
@@ -103,6 +106,7 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
             bool ok = true;
             for (int m = 0; m < 2 && ok; ++m) {
                 if (n_rows[m] <= 0) continue;
+                const int row_begin = row_begin_m[m], row_end = row_end_m[m];
                 const CUtensorMap *tA = m ? &tmA1 : &tmA0;
                 const CUtensorMap *tW = m ? &tmW1 : &tmW0;
                 const CUtensorMap *tP = m ? &tmP1 : &tmP0;
@@ -147,6 +151,7 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
             const uint32_t idesc = umma_idesc_bf16_m128(kSmallN);
             for (int m = 0; m < 2 && ok; ++m) {
                 if (n_rows[m] <= 0) continue;
+                const int row_begin = row_begin_m[m], row_end = row_end_m[m];
                 const int kblocks = (p.H[m] + kSmallBlockK - 1) / kSmallBlockK;
                 for (int row0 = row_begin; row0 < row_end && ok; row0 += kSmallTileRows, ++tc) {
                     const uint32_t buf = tc & 1u;
@@ -188,6 +193,7 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
         bool ok = true;
         for (int m = 0; m < 2 && ok; ++m) {
             if (n_rows[m] <= 0) continue;
+            const int row_begin = row_begin_m[m], row_end = row_end_m[m];
             float sm[NB], ss[NB], stt[NB];
             int sidx[NB];
 #pragma unroll
@@ -223,7 +229,7 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[buf]));
                 const int r_in = quad * 32 + lane;
                 const int row = row0 + r_in;                       // vocabulary entry of this thread
-                if (r_in < nrows && row < p.V) {
+                if (r_in < nrows && row < p.V[m]) {
 #pragma unroll
                     for (int j = 0; j < NB; ++j) {
                         const float z = v[j];

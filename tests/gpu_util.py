@@ -30,7 +30,8 @@ class GpuGate:
                                 start_model=cfg.start_model, W_small=self.W_small,
                                 W_large=self.W_large, device=torch.cuda.current_device(),
                                 stream=self.stream.cuda_stream, temperature=temperature, seed=seed,
-                                eos_token=eos_token)
+                                eos_token=eos_token,
+                                V_large=0 if W_large_bits.shape[0] == cfg.V else W_large_bits.shape[0])
 
     def close(self):
         if self.ctx:

@@ -273,3 +273,35 @@ def test_end_of_sequence_token_and_done_mask(B, V):
     assert np.all(one["tok"][:, 1] == -1) and np.all(np.isnan(one["H"][:, 1]))
     assert np.array_equal(one["tok"][:, 0], free["tok"][:3, 0])
     assert len(blob) > 0
+
+
+@pytest.mark.parametrize("B,Vs,Vl", [(3, 1000, 1700), (40, 2100, 900), (16, 257, 4100)])
+def test_different_vocabularies_per_model(B, Vs, Vl):
+    cfg = _cfg(B=B, V=Vs, T=20, tau=0.5 * (_mid_tau(Vs) + _mid_tau(Vl)))
+    wl = synth.Workload(cfg)
+    W_large = synth.lm_head(cfg.seed + 1, 1, Vl, cfg.H_large)
+    ora = O.run(wl.W_small, W_large, wl.h_small, wl.h_large, w=cfg.w, d_min=cfg.d_min,
+                tau=float(np.float32(cfg.tau)))
+    with GpuGate(cfg, wl.W_small, W_large) as g:
+        out = g.run(wl.h_small, wl.h_large, "run")
+    compare(out, ora, cfg.tau)
+    assert 0.02 < out["used"].mean() < 0.98
+    assert out["tok"][out["used"] == 0].max() < Vs and out["tok"][out["used"] == 1].max() < Vl
+
+
+def test_paper_threshold_grid_in_bits():
+    """The paper's thresholds (bits, Table 1's tau column) on the tiny workload: usage grows as tau
+    falls, tau = 99 never leaves the small model and tau = 0 leaves it after d_min tokens."""
+    from workloads import configs
+    cfg0 = configs.TINY.with_(unit=1)
+    wl = synth.Workload(cfg0)
+    shares = []
+    for tau in (99.0, 1.0, 0.5, 0.25, 0.125, 0.0625, 0.03125, 0.0):
+        cfg = cfg0.with_(tau=tau)
+        with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+            out = g.run(wl.h_small, wl.h_large, "run")
+            use = g.E.ead_usage(g.ctx)
+        shares.append(use["tokens_large"] / (use["tokens_small"] + use["tokens_large"]))
+        assert out["used"].mean() == pytest.approx(shares[-1])
+    assert shares[0] == 0.0 and shares[-1] == pytest.approx((cfg0.T - 10) / cfg0.T)
+    assert all(a <= b for a, b in zip(shares, shares[1:]))

@@ -444,3 +444,24 @@ def test_end_of_sequence_token_stops_a_row_and_only_that_row():
             assert np.all(out["used"][stop:, b] == full["next"][stop - 1, b])
             assert np.all(out["next"][stop:, b] == full["next"][stop - 1, b])
             assert np.all(out["c_after"][stop:, b] == full["c_after"][stop - 1, b])
+
+
+# ---------------------------------------------------------------- two vocabularies
+def test_run_with_different_vocabularies_per_model():
+    """The models may be of different architectures: each step's logits, entropy and token
+    live in the vocabulary of the model that produced them."""
+    r, Ws, _, hs, hl = _tiny_inputs(V=300)
+    Wl = synth.lm_head(78, 1, 520, hl.shape[2])
+    out = O.run(Ws, Wl, hs, hl, w=3, d_min=2, tau=4.9)
+    assert 0 < out["used"].mean() < 1
+    T, B = r.shape
+    for t in range(T):
+        for b in range(B):
+            if out["used"][t, b] == 0:
+                z = O.logits(Ws, hs[t, b])
+                assert z.size == 300
+            else:
+                z = O.logits(Wl, hl[t, b])
+                assert z.size == 520
+            assert out["H"][t, b] == O.entropy(z) and out["tok"][t, b] == O.greedy(z)[0]
+    assert out["tok"][out["used"] == 1].max() >= 300       # tokens beyond the small vocabulary occur
