@@ -269,7 +269,7 @@ def run_ours(args, cfg):
                 "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES_PER_LAUNCH.get(cfg.name)
-    roof.update({"kernel": "ead_lmhead_small_kernel" if B <= 16 else "ead_lmhead_kernel", "kernel_us_per_launch": t_kernel * 1e6,
+    roof.update({"kernel": "ead_lmhead_small_kernel" if B <= 128 else "ead_lmhead_kernel", "kernel_us_per_launch": t_kernel * 1e6,
                  "algorithmic_bytes_per_launch": bytes_s.mean(), "flops_per_launch": flops_s.mean(),
                  "peak_source": peaks["source"] + (" (sustained bf16)" if roof["bound"] == "tensor" else ""),
                  "step_frac": (bytes_s.mean() / (t_ms * 1e-3 / K) / 1e9 / peaks["hbm_gbs"]) if roof["bound"] == "hbm"

@@ -21,6 +21,7 @@ using namespace ead;
 
 namespace {
 
+constexpr int kMidCols = 32;              // value of ead_ctx::small_cols that selects ead_lmhead_small_kernel<0>
 constexpr int kGraphChunk = 32;           // gate steps unrolled in the replayed graph
 constexpr uint32_t kStateMagic = 0x45414433u;   // "EAD3"
 constexpr size_t kHostStageBytes = 64u << 20;   // per staging buffer of ead_run_host
@@ -71,7 +72,8 @@ struct ead_ctx {
     cudaStream_t cap_stream = nullptr;     // capture happens on a private stream
     int G = 0, a_rows = 0, stages = 0, slots_stride = 0;
     int V_large = 0;                       // vocabulary of the large head (cfg.V_large, or cfg.V if that is 0)
-    int small_cols = 0;                    // > 0: swapped-operand kernel with this many batch columns
+    int small_cols = 0;                    // > 0: swapped-operand kernel: batch columns per thread (1..16), or
+                                           // kMidCols for its 17..128-sequence variant
     int small_slots = 0;                   // partial slots per row it writes (one per CTA and epilogue warp)
     size_t smem_bytes = 0;
     const void *W[2] = {nullptr, nullptr};
@@ -182,7 +184,8 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
         case 2: EAD_LAUNCH_SMALL(2); break;
         case 4: EAD_LAUNCH_SMALL(4); break;
         case 8: EAD_LAUNCH_SMALL(8); break;
-        default: EAD_LAUNCH_SMALL(16); break;
+        case 16: EAD_LAUNCH_SMALL(16); break;
+        default: EAD_LAUNCH_SMALL(0); break;     // kMidCols
     }
 #undef EAD_LAUNCH_SMALL
     if (e != cudaSuccess) return EAD_ECUDA;
@@ -404,12 +407,21 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
         stage_bytes = small_stage_bytes(x->a_rows);
         x->small_slots = x->G * kSmallSlotsPerCta;
         x->slots_stride = (x->small_slots + 31) & ~31;
+    } else if (cfg->B <= kMidMaxRows) {
+        // still bound by streaming the weights: same kernel, sequences in chunks of 32
+        x->small_cols = kMidCols;
+        x->a_rows = (cfg->B + 15) / 16 * 16;
+        stage_bytes = small_stage_bytes(x->a_rows);
+        x->small_slots = x->G * kSmallSlotsPerCta;
+        x->slots_stride = (x->small_slots + 31) & ~31;
     } else {
         x->a_rows = std::min(kTileM, (cfg->B + 7) & ~7);
         stage_bytes = static_cast<size_t>(x->a_rows) * kBlockK * 2 + kWTileBytes;
     }
-    x->stages = static_cast<int>(std::min<size_t>(kMaxStages, (smem_max - kSmemCtrlBytes - 1024 - 1024) / stage_bytes));
-    x->smem_bytes = kSmemCtrlBytes + 1024 + x->stages * stage_bytes;
+    const size_t extra = x->small_cols == kMidCols ? kTransposeBytes : 0;   // transpose tiles of its epilogue
+    x->stages = static_cast<int>(
+        std::min<size_t>(kMaxStages, (smem_max - kSmemCtrlBytes - 1024 - 1024 - extra) / stage_bytes));
+    x->smem_bytes = kSmemCtrlBytes + 1024 + x->stages * stage_bytes + extra;
 
     const int B = cfg->B;
     // compacted operands are padded to whole row blocks (zeros) so that no TMA box of
@@ -471,7 +483,9 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
         reinterpret_cast<const void *>(ead_lmhead_small_kernel<2, true>),
         reinterpret_cast<const void *>(ead_lmhead_small_kernel<4, true>),
         reinterpret_cast<const void *>(ead_lmhead_small_kernel<8, true>),
-        reinterpret_cast<const void *>(ead_lmhead_small_kernel<16, true>)};
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<16, true>),
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<0, false>),
+        reinterpret_cast<const void *>(ead_lmhead_small_kernel<0, true>)};
     for (const void *k : lmhead_kernels) {
         cudaFuncAttributes fa;
         if (cudaFuncGetAttributes(&fa, k) != cudaSuccess) return fail(EAD_ECUDA);

@@ -14,6 +14,7 @@ constexpr int kMaxStages = 8;
 constexpr int kMaxCtas = 256;         // upper bound on the LM-head grid (one CTA per SM)
 constexpr int kWTileBytes = kTileN * kBlockK * 2;   // 32 KiB
 constexpr int kSmemCtrlBytes = 1024;
+constexpr int kTransposeBytes = 4 * 32 * 33 * 4;    // four 32 x 33 float tiles (one per epilogue warp)
 constexpr int kLmheadThreads = 192;                 // TMA warp, MMA warp, 4 epilogue warps
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kNegSentinel = -1.0e30f;            // "no logit seen yet"; finite on purpose

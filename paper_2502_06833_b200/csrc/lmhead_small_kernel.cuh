@@ -24,6 +24,13 @@
 // the MMA's N = 16 then reads the following kilobyte as rows 8-15, which only feeds
 // accumulator columns nobody reads).  TMEM holds two 16-column accumulators so that the
 // epilogue overlaps the next tile's MMAs.
+//
+// NB = 0 selects the variant for 17..128 sequences: the MMA's N is the number of active rows
+// of the head rounded up to 16 (<= 128), the accumulators are 128 columns apart, and the
+// epilogue cannot keep one statistic per sequence in registers any more.  Instead each warp
+// transposes its 32 vocabulary rows x 32 sequences through a private shared-memory tile, after
+// which lane l holds 32 consecutive logits of sequence (chunk * 32 + l) and folds them with the
+// same 32-column routine as the large-batch kernel.
 #pragma once
 #include "lmhead_kernel.cuh"
 
@@ -35,7 +42,7 @@ constexpr int kSmallSlotsPerCta = 4;                   // one partial per epilog
 constexpr int kSmallN = 16;                            // batch columns (MMA N)
 constexpr int kSmallBlockK = 128;                      // hidden elements per stage
 constexpr int kSmallWBytes = kSmallTileRows * 64 * 2;  // one 64-wide box of W rows: 16 KiB
-constexpr int kSmallTmemCols = 32;                     // 2 accumulators x 16 columns
+constexpr int kMidMaxRows = 128;                       // largest batch of the NB = 0 variant
 __host__ __device__ constexpr int small_stage_bytes(int h_rows) { return 2 * h_rows * 128 + 2 * kSmallWBytes; }
 
 template <int NB, bool SAMPLE>
@@ -57,6 +64,8 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
     const int stages = p.stages;
     const uint32_t h_slab = static_cast<uint32_t>(p.a_rows) * 128;      // hidden rows of one 64-wide K slab
     const uint32_t stage_bytes = 2 * h_slab + 2 * kSmallWBytes;
+    constexpr uint32_t kAccCols = NB == 0 ? 128u : static_cast<uint32_t>(kSmallN);   // TMEM columns per accumulator
+    float *trans = reinterpret_cast<float *>(stage0 + static_cast<size_t>(stages) * stage_bytes);   // NB = 0 only
     StepCtl *ctl = p.ctl_rw;
 
     if (threadIdx.x == 0) {
@@ -78,7 +87,7 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
         tma_prefetch_desc(&tmP0); tma_prefetch_desc(&tmP1);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(&ctrl->tmem_base), kSmallTmemCols);
+        tmem_alloc(smem_u32(&ctrl->tmem_base), 2 * kAccCols);
         tmem_relinquish();
     }
     tc_fence_before_sync();
@@ -148,11 +157,12 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
         if (lane == 0) {
             uint32_t it = 0, tc = 0;
             bool ok = true;
-            const uint32_t idesc = umma_idesc_bf16_m128(kSmallN);
             for (int m = 0; m < 2 && ok; ++m) {
                 if (n_rows[m] <= 0) continue;
                 const int row_begin = row_begin_m[m], row_end = row_end_m[m];
                 const int kblocks = (p.H[m] + kSmallBlockK - 1) / kSmallBlockK;
+                const uint32_t idesc =
+                    umma_idesc_bf16_m128(NB == 0 ? static_cast<uint32_t>((n_rows[m] + 15) / 16 * 16) : kSmallN);
                 for (int row0 = row_begin; row0 < row_end && ok; row0 += kSmallTileRows, ++tc) {
                     const uint32_t buf = tc & 1u;
                     if (!wait_bar(smem_u32(&ctrl->tmem_empty[buf]), ((tc >> 1) & 1u) ^ 1u, ctrl, ctl)) {
@@ -160,7 +170,7 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                         break;
                     }
                     tc_fence_after_sync();
-                    const uint32_t d_tmem = tmem_base + buf * kSmallN;
+                    const uint32_t d_tmem = tmem_base + buf * kAccCols;
                     for (int kb = 0; kb < kblocks; ++kb, ++it) {
                         const uint32_t s = it % stages;
                         if (!wait_bar(smem_u32(&ctrl->full[s]), (it / stages) & 1u, ctrl, ctl)) {
@@ -194,6 +204,73 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
         for (int m = 0; m < 2 && ok; ++m) {
             if (n_rows[m] <= 0) continue;
             const int row_begin = row_begin_m[m], row_end = row_end_m[m];
+            if constexpr (NB == 0) {
+                float *tbuf = trans + quad * (32 * 33);
+                const int n16 = (n_rows[m] + 15) / 16 * 16;
+                const int nch = (n16 + 31) / 32;                    // <= 4 chunks of 32 sequences
+                const uint32_t rng_step = static_cast<uint32_t>(p.ctl->cur_t);
+                RowStat st3[4];
+                Draw dr3[4];
+                uint32_t rr3[4];
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    rowstat_reset(st3[ch]);
+                    dr3[ch] = Draw{-INFINITY, 0x7fffffff};
+                    const int j = ch * 32 + lane;
+                    rr3[ch] = (SAMPLE && j < n_rows[m]) ? static_cast<uint32_t>(p.perm[m * p.B + j]) : 0u;
+                }
+                for (int row0 = row_begin; row0 < row_end && ok; row0 += kSmallTileRows, ++tc) {
+                    const int nrows = min(kSmallTileRows, row_end - row0);
+                    const uint32_t buf = tc & 1u;
+                    if (!wait_bar_warp(smem_u32(&ctrl->tmem_full[buf]), (tc >> 1) & 1u, ctrl, ctl, lane)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const int cb = row0 + quad * 32;                // vocabulary entries held by this warp's lanes
+                    const int limit = min(p.V[m], row0 + nrows);    // first invalid vocabulary entry of the tile
+                    if (cb < limit) {
+                        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + buf * kAccCols;
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) {
+                            if (ch >= nch) continue;
+                            float v[32], w[32];
+                            tmem_ld_32cols(taddr + ch * 32, v);
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) tbuf[j * 33 + lane] = v[j];
+                            __syncwarp();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) w[i] = tbuf[lane * 33 + i];
+                            __syncwarp();
+                            if (cb + 32 > limit) {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) w[i] = (cb + i < limit) ? w[i] : kNegSentinel;
+                            }
+                            rowstat_absorb32(st3[ch], w, cb);
+                            if (SAMPLE) draw_absorb32(dr3[ch], w, cb, rng_step, rr3[ch], p);
+                            __syncwarp();
+                        }
+                    }
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[buf]));
+                }
+                if (!ok) break;
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    const int j = ch * 32 + lane;
+                    if (ch >= nch || j >= n_rows[m]) continue;
+                    const size_t o = (static_cast<size_t>(m) * p.B + j) * p.slots_stride + cta * kSmallSlotsPerCta + quad;
+                    p.part_m[o] = st3[ch].m;
+                    p.part_s[o] = st3[ch].s;
+                    p.part_t[o] = st3[ch].t;
+                    p.part_i[o] = st3[ch].idx;
+                    if (SAMPLE) {
+                        p.part_k[o] = dr3[ch].k;
+                        p.part_ki[o] = dr3[ch].ki;
+                    }
+                }
+            } else {
             float sm[NB], ss[NB], stt[NB];
             int sidx[NB];
 #pragma unroll
@@ -298,13 +375,14 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                     }
                 }
             }
+            }
         }
     }
 
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    if (warp == 1) tmem_dealloc(tmem_base, kSmallTmemCols);
+    if (warp == 1) tmem_dealloc(tmem_base, 2 * kAccCols);
 }
 
 }  // namespace ead

@@ -42,6 +42,8 @@ SHAPES = [
     (130, 3000, 64, 128),         # two row blocks, the second with 2 rows
     (300, 5000, 128, 256),        # three row blocks shared by both heads
     (128, 2048, 64, 64),          # exactly one full row block
+    (100, 2300, 128, 64),         # four chunks of sequences in the 17..128 variant, the last ragged
+    (17, 700, 64, 128),           # smallest batch of that variant
 ]
 
 
@@ -224,7 +226,7 @@ def test_usage_counters_follow_the_trace_and_survive_a_checkpoint():
 
 @pytest.mark.parametrize("B,V,Hs,Hl,temp", [(3, 1000, 64, 128, 1.0), (1, 4100, 256, 512, 0.7),
                                             (12, 2500, 128, 64, 1.5), (40, 3000, 64, 128, 1.0),
-                                            (130, 1700, 64, 64, 0.8)])
+                                            (97, 1100, 64, 128, 1.2), (130, 1700, 64, 64, 0.8)])
 def test_temperature_sampling_matches_the_oracle_draws(B, V, Hs, Hl, temp):
     """Algorithm 1's sampling lines: same Philox stream and Gumbel-max rule on both sides, so
     the drawn tokens must be identical (up to logged near-ties of the perturbed values);
