@@ -307,3 +307,37 @@ def test_paper_threshold_grid_in_bits():
         assert out["used"].mean() == pytest.approx(shares[-1])
     assert shares[0] == 0.0 and shares[-1] == pytest.approx((cfg0.T - 10) / cfg0.T)
     assert all(a <= b for a, b in zip(shares, shares[1:]))
+
+
+def test_two_contexts_of_different_shape_interleaved_on_a_side_stream():
+    """Contexts with different pipelines (stage counts, kernels) coexist and do not disturb each
+    other; a non-default stream works."""
+    import torch
+    cfg_a = _cfg(B=3, V=1100, T=12, tau=_mid_tau(1100))
+    cfg_b = _cfg(B=140, V=900, H_small=128, H_large=64, T=12, tau=_mid_tau(900), seed=9)
+    wa, wb = synth.Workload(cfg_a), synth.Workload(cfg_b)
+    oa, ob = _oracle(cfg_a, wa), _oracle(cfg_b, wb)
+    side = torch.cuda.Stream()
+    with GpuGate(cfg_b, wb.W_small, wb.W_large, stream=side) as gb, GpuGate(cfg_a, wa.W_small, wa.W_large) as ga:
+        outs_a, outs_b = [], []
+        for t0 in range(0, 12, 4):                       # alternate between the two contexts
+            outs_a.append(ga.run(wa.h_small[t0:t0 + 4], wa.h_large[t0:t0 + 4], "run"))
+            outs_b.append(gb.run(wb.h_small[t0:t0 + 4], wb.h_large[t0:t0 + 4], "run"))
+    cat = lambda outs: {k: np.concatenate([o[k] for o in outs]) for k in outs[0]}
+    compare(cat(outs_a), oa, cfg_a.tau)
+    compare(cat(outs_b), ob, cfg_b.tau)
+
+
+def test_host_entry_point_over_several_staging_chunks():
+    """ead_run_host stages the hidden states in chunks (64 MB per buffer): a run longer than one
+    chunk must give what the device-resident run gives."""
+    cfg = _cfg(B=48, V=320, H_small=4096, H_large=4096, T=190, tau=_mid_tau(320), d_min=3)
+    wl = synth.Workload(cfg)                             # 48 * 8192 * 2 B = 768 KB per step: 85 steps per chunk
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        a = g.run(wl.h_small, wl.h_large, "run")
+        g.E.ead_reset(g.ctx)
+        b = g.run(wl.h_small, wl.h_large, "host")
+    for k in ("tok", "H", "Hbar", "used", "next"):
+        assert np.array_equal(a[k], b[k]), k
+    ora = _oracle(cfg, wl, T=40)
+    compare({k: v[:40] for k, v in a.items()}, ora, cfg.tau)
