@@ -52,6 +52,7 @@ extern "C" {
 #define EAD_STATUS_NONFINITE   0x1u /* some row saw a NaN / infinite logit (row gets H = NaN) */
 #define EAD_STATUS_WAIT_EXPIRED 0x2u /* a bounded wait inside a kernel ran out                 */
 #define EAD_STATUS_BAD_COUNT   0x4u /* internal row counts inconsistent                       */
+#define EAD_STATUS_SHARD_MISMATCH 0x8u /* vocabulary shards disagree on the step or on a row's model */
 
 typedef struct ead_ctx ead_ctx; /* opaque */
 
@@ -75,6 +76,12 @@ typedef struct ead_config {
     int32_t V_large;     /* vocabulary of M_L if it differs from V (the paper allows models of
                             different architectures); 0 = same as V.  Tokens of a step are
                             indices into the vocabulary of the model that produced them      */
+    int32_t shard_count; /* 0: this context holds the whole heads.  n >= 1: it holds one of n
+                            vocabulary slices (see ead_shard_connect); V and V_large are then the
+                            rows of its slices                                                   */
+    int32_t vocab_offset_small; /* sharded: row of the full small head at which this slice starts,
+                                   a multiple of 16; tokens are reported in full-head indices   */
+    int32_t vocab_offset_large; /* the same for the large head                                  */
 } ead_config;
 
 /*
@@ -152,7 +159,8 @@ int ead_reset(ead_ctx *ctx);
 
 /* Waits for the context's stream, then reports the device status word
  * (EAD_STATUS_* bits, sticky until ead_reset).  Returns EAD_EDEVICE_FAULT if
- * EAD_STATUS_WAIT_EXPIRED or EAD_STATUS_BAD_COUNT is set, else EAD_OK. */
+ * EAD_STATUS_WAIT_EXPIRED or EAD_STATUS_BAD_COUNT is set, EAD_ESTATE if
+ * EAD_STATUS_SHARD_MISMATCH is set, else EAD_OK. */
 int ead_status(ead_ctx *ctx, uint32_t *status_word);
 
 /*
@@ -203,6 +211,76 @@ int64_t ead_kernel_launches(const ead_ctx *ctx);
  * {CTAs of the LM-head kernel, pipeline stages, rows of the hidden-state TMA
  * box, dynamic shared memory bytes}. */
 int ead_launch_info(const ead_ctx *ctx, int32_t *info, int32_t n);
+
+/*
+ * Vocabulary-sharded gate step (several GPUs, one sequence batch).  The softmax of Eq. 1 and
+ * the entropy of Eq. 2 are sums over the vocabulary and the greedy / sampled token is a maximum
+ * over it, so the vocabulary rows of both heads can be split over n GPUs: each computes the
+ * statistics of its slice, the slices' statistics are exchanged (n x B records of 32 bytes:
+ * the only traffic between the GPUs), and every GPU merges all of them in shard order and runs
+ * the window / dwell / threshold part of Algorithm 1 itself.  All GPUs then hold identical
+ * per-sequence state and identical outputs, bit for bit, without further communication.  The
+ * paper describes one device; this split is the build's own.
+ *
+ * Each GPU creates a context with cfg.shard_count = n (<= 16), cfg.V / cfg.V_large = rows of its
+ * slices, cfg.vocab_offset_* = where they start, and the slice pointers as W_small / W_large;
+ * all other fields equal on all GPUs.  Every GPU gets the full hidden rows at every step.
+ *
+ * ead_shard_range: the slice [*begin, *end) of a head of V rows that shard `shard` of n_shards
+ * takes when the rows are dealt out in whole tiles of 128 (host arithmetic, needs no GPU).
+ * Errors: EAD_EINVALID_ARG (also when n_shards exceeds the number of tiles).
+ *
+ * The exchange can run in two ways.
+ *
+ * (1) Inside the kernels, over peer memory.  Every shard owns an exchange buffer of
+ * ead_shard_exchange_bytes(B, n) bytes, zero-filled, 16-byte aligned, mapped into the address
+ * space of every other shard's GPU (peer access, an IPC handle, symmetric memory).
+ *     ead_shard_connect(ctx, shard, exchange)   exchange: host array [n]; entry d = shard d's
+ *                                               buffer as addressable from this GPU (entry
+ *                                               `shard` is this context's own, local buffer)
+ * From then on ead_step / ead_run / ead_run_host work as on one GPU, called on every shard with
+ * the same hidden states: after its cross-CTA merge each shard stores its B records straight
+ * into all n exchange buffers (plain stores; the record's step word last, with release
+ * semantics at system scope), and a fourth kernel waits until the records of all n shards for
+ * this step have arrived in the local buffer and finishes the step.  Buffers alternate with
+ * the parity of the step, which suffices because a shard cannot run more than one step ahead
+ * of another.  The wait is bounded (2 s): a shard that never delivers sets
+ * EAD_STATUS_WAIT_EXPIRED, the rows are reported like non-finite rows, and later steps do not
+ * wait again.  Waits for the stream; restarts the numbering of exchanged records, so all shards
+ * connect (to zero-filled buffers) at the same point of their runs.  ead_reset, ead_set_state
+ * and ead_set_done must be applied on all shards alike.
+ * Errors: EAD_EINVALID_ARG, EAD_EALIGNMENT, EAD_ECUDA.  Before ead_shard_connect the stepping
+ * calls return EAD_EINVALID_ARG on a sharded context; ead_run_timed always does.
+ *
+ * (2) By the caller, between two library calls (NCCL or any other all-gather that is ordered
+ * on the context's stream); no peer mapping needed:
+ *     ead_shard_partials(ctx, h_small, h_large, records);      // this GPU's [B] records
+ *     <all-gather the n record arrays, in shard order, into all_records on every GPU>
+ *     ead_shard_gate(ctx, all_records, n, tok, H, Hbar, model_used, next_model);
+ *   records      dev, [B] x EAD_SHARD_RECORD_BYTES, 16-byte aligned: per sequence (caller's row
+ *                order) {float m, s, t; int32 idx; float k; int32 ki; int32 model; int32 step1}:
+ *                max, sum exp(z - m), sum exp(z - m)(z - m) log2 e and arg max of the slice's
+ *                logits, the sampling candidate, the head they belong to, and 1 + the number
+ *                of sharded steps this context has taken.  Rows of ended sequences are not
+ *                written.
+ *   all_records  dev, [n_shards][B] records, shard s at index s
+ *   outputs      as in ead_step
+ * Both calls are asynchronous on the context's stream.  On a connected context `records` and
+ * `all_records` may be NULL: the two halves of a step of way (1), called apart.
+ *
+ * In both ways a record whose model or step number differs from this context's sets
+ * EAD_STATUS_SHARD_MISMATCH and leaves the row's state untouched (outputs as for a non-finite
+ * row).  Errors of (2): EAD_EINVALID_ARG (also: context not created with shard_count >= 1, or
+ * n_shards not equal to it), EAD_EALIGNMENT, EAD_ECUDA.
+ */
+#define EAD_SHARD_RECORD_BYTES 32
+#define EAD_SHARD_MAX 16
+int ead_shard_range(int32_t V, int32_t n_shards, int32_t shard, int32_t *begin, int32_t *end);
+size_t ead_shard_exchange_bytes(int32_t B, int32_t n_shards);
+int ead_shard_connect(ead_ctx *ctx, int32_t shard, void *const *exchange);
+int ead_shard_partials(ead_ctx *ctx, const void *h_small, const void *h_large, void *records);
+int ead_shard_gate(ead_ctx *ctx, const void *all_records, int32_t n_shards, int32_t *tok, float *H,
+                   float *Hbar, uint8_t *model_used, uint8_t *next_model);
 
 /*
  * How the LM-head kernel divides one head among its CTAs (host-side replica of the rule

@@ -25,11 +25,16 @@ EAD_STATIC_MAX_H = 8192
 EAD_STATUS_NONFINITE = 0x1
 EAD_STATUS_WAIT_EXPIRED = 0x2
 EAD_STATUS_BAD_COUNT = 0x4
+EAD_STATUS_SHARD_MISMATCH = 0x8
+EAD_SHARD_RECORD_BYTES = 32
+EAD_SHARD_MAX = 16
 
 SYMBOLS = ["ead_create", "ead_step", "ead_run", "ead_run_host", "ead_run_timed", "ead_reset", "ead_status",
            "ead_state_size", "ead_get_state", "ead_set_state", "ead_kernel_launches",
            "ead_launch_info", "ead_destroy", "ead_strerror", "ead_head_entropy_static",
-           "ead_plan_split", "ead_usage", "ead_parameter_ratio", "ead_set_done", "ead_get_done"]
+           "ead_plan_split", "ead_usage", "ead_parameter_ratio", "ead_set_done", "ead_get_done",
+           "ead_shard_range", "ead_shard_partials", "ead_shard_gate", "ead_shard_connect",
+           "ead_shard_exchange_bytes"]
 
 
 class EadConfig(C.Structure):
@@ -37,7 +42,8 @@ class EadConfig(C.Structure):
                 ("w", C.c_int32), ("d_min", C.c_int32), ("tau", C.c_float), ("unit", C.c_int32),
                 ("start_model", C.c_int32), ("device", C.c_int32), ("stream", C.c_void_p),
                 ("temperature", C.c_float), ("seed", C.c_uint64), ("eos_token", C.c_int32),
-                ("V_large", C.c_int32)]
+                ("V_large", C.c_int32), ("shard_count", C.c_int32), ("vocab_offset_small", C.c_int32),
+                ("vocab_offset_large", C.c_int32)]
 
 
 class EadError(RuntimeError):
@@ -98,6 +104,16 @@ def lib() -> C.CDLL:
         L.ead_parameter_ratio.argtypes = [C.c_uint64, C.c_uint64, C.c_double, C.c_double]
         L.ead_plan_split.restype = C.c_int
         L.ead_plan_split.argtypes = [C.c_int32] * 4 + [C.POINTER(C.c_int32)]
+        L.ead_shard_range.restype = C.c_int
+        L.ead_shard_range.argtypes = [C.c_int32] * 3 + [C.POINTER(C.c_int32)] * 2
+        L.ead_shard_exchange_bytes.restype = C.c_size_t
+        L.ead_shard_exchange_bytes.argtypes = [C.c_int32, C.c_int32]
+        L.ead_shard_connect.restype = C.c_int
+        L.ead_shard_connect.argtypes = [vp, C.c_int32, C.POINTER(C.c_void_p)]
+        L.ead_shard_partials.restype = C.c_int
+        L.ead_shard_partials.argtypes = [vp, vp, vp, vp]
+        L.ead_shard_gate.restype = C.c_int
+        L.ead_shard_gate.argtypes = [vp, vp, C.c_int32, i32p, f32p, f32p, u8p, u8p]
         L.ead_strerror.restype = C.c_char_p
         L.ead_strerror.argtypes = [C.c_int]
         _lib = L
@@ -125,11 +141,13 @@ def _ptr(t):
 
 
 def ead_create(*, B, V, H_small, H_large, w, d_min, tau, W_small, W_large, unit=0, start_model=0,
-               device=0, stream=0, temperature=0.0, seed=0, eos_token=-1, V_large=0):
+               device=0, stream=0, temperature=0.0, seed=0, eos_token=-1, V_large=0, shard_count=0,
+               vocab_offset_small=0, vocab_offset_large=0):
     """Returns an opaque context handle (int).  ``W_*`` are device bf16 ``[V, H]``; they are
     borrowed, keep them alive until ``ead_destroy``."""
     cfg = EadConfig(B, V, H_small, H_large, w, d_min, float(tau), unit, start_model, device,
-                    C.c_void_p(int(stream)), float(temperature), int(seed), int(eos_token), int(V_large))
+                    C.c_void_p(int(stream)), float(temperature), int(seed), int(eos_token), int(V_large),
+                    int(shard_count), int(vocab_offset_small), int(vocab_offset_large))
     out = C.c_void_p()
     _check(lib().ead_create(C.byref(cfg), _ptr(W_small), _ptr(W_large), C.byref(out)), "ead_create")
     return out.value
@@ -239,6 +257,33 @@ def ead_plan_split(cta, G, n_rows, V) -> dict:
     a = (C.c_int32 * 6)()
     _check(lib().ead_plan_split(int(cta), int(G), int(n_rows), int(V), a), "ead_plan_split")
     return dict(active=a[0], row_block=a[1], slot=a[2], col_begin=a[3], col_end=a[4], group=a[5])
+
+
+def ead_shard_range(V, n_shards, shard) -> tuple:
+    """Rows ``[begin, end)`` of a head of V rows held by ``shard`` of ``n_shards``."""
+    b, e = C.c_int32(), C.c_int32()
+    _check(lib().ead_shard_range(int(V), int(n_shards), int(shard), C.byref(b), C.byref(e)), "ead_shard_range")
+    return int(b.value), int(e.value)
+
+
+def ead_shard_exchange_bytes(B, n_shards) -> int:
+    return int(lib().ead_shard_exchange_bytes(int(B), int(n_shards)))
+
+
+def ead_shard_connect(ctx, shard, exchange) -> None:
+    """``exchange``: one device address (or tensor) per shard, as addressable from this GPU."""
+    ptrs = (C.c_void_p * len(exchange))(*[_ptr(e) for e in exchange])
+    _check(lib().ead_shard_connect(ctx, int(shard), ptrs), "ead_shard_connect")
+
+
+def ead_shard_partials(ctx, h_small, h_large, records) -> None:
+    _check(lib().ead_shard_partials(ctx, _ptr(h_small), _ptr(h_large), _ptr(records)), "ead_shard_partials")
+
+
+def ead_shard_gate(ctx, all_records, n_shards, tok=None, H=None, Hbar=None, model_used=None,
+                   next_model=None) -> None:
+    _check(lib().ead_shard_gate(ctx, _ptr(all_records), int(n_shards), _ptr(tok), _ptr(H), _ptr(Hbar),
+                                _ptr(model_used), _ptr(next_model)), "ead_shard_gate")
 
 
 def ead_destroy(ctx) -> None:

@@ -86,6 +86,8 @@ struct ead_ctx {
     uint32_t *usage = nullptr;
     float *ring = nullptr, *part_m = nullptr, *part_s = nullptr, *part_t = nullptr;
     uint16_t *hc[2] = {nullptr, nullptr};
+    ShardLink *link = nullptr;             // vocabulary-sharded contexts: where the records go (device)
+    bool connected = false;                // ead_shard_connect has filled `link`
     CUtensorMap tmA[2], tmW[2], tmT[2], tmP[2];   // hidden rows; W boxes of 256|128, 16 and 32 rows
     cudaGraphExec_t g_one = nullptr, g_chunk = nullptr;
     int64_t launches = 0;
@@ -129,10 +131,50 @@ cudaError_t launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+GateParams gate_params(const ead_ctx *x, int reduce_only)
+{
+    const ead_config &c = x->cfg;
+    GateParams gp{};
+    gp.B = c.B;
+    gp.V = c.V;
+    gp.w = c.w;
+    gp.d_min = c.d_min;
+    gp.unit = c.unit;
+    gp.G = x->G;
+    gp.slots_stride = x->slots_stride;
+    gp.n_slots = x->small_slots;
+    gp.tau = c.tau;
+    gp.ctl = x->ctl;
+    gp.args = x->args;
+    gp.part_m = x->part_m;
+    gp.part_s = x->part_s;
+    gp.part_t = x->part_t;
+    gp.part_i = x->part_i;
+    gp.sampling = c.temperature > 0.f ? 1 : 0;
+    gp.part_k = x->part_k;
+    gp.part_ki = x->part_ki;
+    gp.perm = x->perm;
+    gp.flag = x->flag;
+    gp.c = x->c;
+    gp.nfill = x->nfill;
+    gp.ring = x->ring;
+    gp.usage = x->usage;
+    gp.done = x->done;
+    gp.eos_token = c.eos_token;
+    gp.reduce_only = reduce_only;
+    gp.link = x->link;
+    gp.v_off[0] = c.vocab_offset_small;
+    gp.v_off[1] = c.vocab_offset_large;
+    return gp;
+}
+
 // The three kernels of one gate step, in stream order.  With `ev` (4 events) the
 // boundaries between the kernels are recorded for timing and the kernels do not overlap;
 // otherwise each kernel's set-up overlaps the tail of the one before it.
-int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
+// shard_mode (vocabulary-sharded contexts): 1 = stop after the merge, records to the caller's
+// buffer; 2 = records into every shard's exchange buffer, then a fourth kernel that waits for
+// all shards' records and finishes the step; 3 = as 2 without the fourth kernel.
+int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr, int shard_mode = 0)
 {
     const ead_config &c = x->cfg;
     const bool pdl = ev == nullptr;
@@ -167,6 +209,8 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     lp.part_k = x->part_k;
     lp.part_ki = x->part_ki;
     lp.perm = x->perm;
+    lp.ctr_off[0] = static_cast<uint32_t>(c.vocab_offset_small) >> 2;
+    lp.ctr_off[1] = static_cast<uint32_t>(c.vocab_offset_large) >> 2;
     const dim3 lgrid(x->G), lblock(kLmheadThreads);
 #define EAD_LAUNCH_SMALL(NB)                                                                                   \
     e = lp.sampling ? launch(ead_lmhead_small_kernel<NB, true>, lgrid, lblock, x->smem_bytes, s, pdl, x->tmA[0],  \
@@ -191,33 +235,7 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
     if (e != cudaSuccess) return EAD_ECUDA;
     if (ev) cudaEventRecord(ev[2], s);
 
-    GateParams gp{};
-    gp.B = c.B;
-    gp.V = c.V;
-    gp.w = c.w;
-    gp.d_min = c.d_min;
-    gp.unit = c.unit;
-    gp.G = x->G;
-    gp.slots_stride = x->slots_stride;
-    gp.n_slots = x->small_slots;
-    gp.tau = c.tau;
-    gp.ctl = x->ctl;
-    gp.args = x->args;
-    gp.part_m = x->part_m;
-    gp.part_s = x->part_s;
-    gp.part_t = x->part_t;
-    gp.part_i = x->part_i;
-    gp.sampling = c.temperature > 0.f ? 1 : 0;
-    gp.part_k = x->part_k;
-    gp.part_ki = x->part_ki;
-    gp.perm = x->perm;
-    gp.flag = x->flag;
-    gp.c = x->c;
-    gp.nfill = x->nfill;
-    gp.ring = x->ring;
-    gp.usage = x->usage;
-    gp.done = x->done;
-    gp.eos_token = c.eos_token;
+    const GateParams gp = gate_params(x, shard_mode == 3 ? 2 : shard_mode);
     const int rows_per_block = kGateThreads / 32;
     if (x->small_cols)
         e = launch(ead_merge_gate_wide_kernel, dim3(c.B), dim3(kGateThreads), 0, s, pdl, gp);
@@ -226,15 +244,25 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr)
                    pdl, gp);
     if (e != cudaSuccess) return EAD_ECUDA;
     if (ev) cudaEventRecord(ev[3], s);
+    if (shard_mode == 2) {
+        e = launch(ead_shard_gate_kernel, dim3((c.B + 127) / 128), dim3(128), 0, s, pdl, gate_params(x, 0),
+                   static_cast<const ShardRecord *>(nullptr), 0, RunArgs{}, 2);
+        if (e != cudaSuccess) return EAD_ECUDA;
+    }
     return cudaGetLastError() == cudaSuccess ? EAD_OK : EAD_ECUDA;
 }
+
+int step_mode(const ead_ctx *x) { return x->cfg.shard_count > 0 ? 2 : 0; }
+int kernels_per_step(const ead_ctx *x) { return x->cfg.shard_count > 0 ? 4 : 3; }
+// Sharded contexts take whole steps only once their exchange buffers are known.
+bool can_step(const ead_ctx *x) { return x->cfg.shard_count == 0 || x->connected; }
 
 int build_graph(ead_ctx *x, int steps, cudaGraphExec_t *out)
 {
     cudaGraph_t graph = nullptr;
     EAD_CUDA(cudaStreamBeginCapture(x->cap_stream, cudaStreamCaptureModeThreadLocal));
     int rc = EAD_OK;
-    for (int i = 0; i < steps && rc == EAD_OK; ++i) rc = enqueue_step(x, x->cap_stream);
+    for (int i = 0; i < steps && rc == EAD_OK; ++i) rc = enqueue_step(x, x->cap_stream, nullptr, step_mode(x));
     cudaError_t e = cudaStreamEndCapture(x->cap_stream, &graph);
     if (rc != EAD_OK || e != cudaSuccess || !graph) {
         if (graph) cudaGraphDestroy(graph);
@@ -251,9 +279,10 @@ int build_graph(ead_ctx *x, int steps, cudaGraphExec_t *out)
 }
 
 int set_args(ead_ctx *x, const void *hs, const void *hl, int32_t *tok, float *H, float *Hbar, uint8_t *used,
-             uint8_t *next, cudaStream_t s)
+             uint8_t *next, cudaStream_t s, float *shard_out = nullptr)
 {
     RunArgs a{};
+    a.shard_out = shard_out;
     a.h[0] = static_cast<const uint16_t *>(hs);
     a.h[1] = static_cast<const uint16_t *>(hl);
     a.tok = tok;
@@ -280,7 +309,7 @@ int run_device(ead_ctx *x, int T, const void *hs, const void *hl, int32_t *tok, 
         EAD_CUDA(cudaGraphLaunch(x->g_one, x->stream));
         left -= 1;
     }
-    x->launches += 3ll * T;
+    x->launches += static_cast<int64_t>(kernels_per_step(x)) * T;
     return EAD_OK;
 }
 
@@ -371,9 +400,14 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
     *out = nullptr;
     if (cfg->B < 1 || cfg->B > 4096 || cfg->V < 1 || cfg->H_small < 8 || cfg->H_large < 8 || cfg->w < 1 ||
         cfg->w > 64 || (cfg->unit != 0 && cfg->unit != 1) || (cfg->start_model != 0 && cfg->start_model != 1) ||
-        !(cfg->temperature >= 0.f) || !(cfg->temperature < 3.0e38f) || cfg->V_large < 0 ||
-        cfg->eos_token >= std::min(cfg->V, cfg->V_large > 0 ? cfg->V_large : cfg->V))
+        !(cfg->temperature >= 0.f) || !(cfg->temperature < 3.0e38f) || cfg->V_large < 0 || cfg->shard_count < 0 ||
+        cfg->shard_count > kMaxShards ||
+        cfg->vocab_offset_small < 0 || cfg->vocab_offset_large < 0 ||
+        (cfg->shard_count == 0 && (cfg->vocab_offset_small || cfg->vocab_offset_large)) ||
+        // a sharded context sees one slice: the end-of-sequence token indexes the full vocabulary
+        (cfg->shard_count == 0 && cfg->eos_token >= std::min(cfg->V, cfg->V_large > 0 ? cfg->V_large : cfg->V)))
         return EAD_EINVALID_ARG;
+    if (cfg->vocab_offset_small % kUnit || cfg->vocab_offset_large % kUnit) return EAD_EALIGNMENT;
     if (cfg->H_small % 8 || cfg->H_large % 8 || !aligned16(W_small) || !aligned16(W_large)) return EAD_EALIGNMENT;
 
     int ndev = 0;
@@ -446,6 +480,10 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
         cudaMalloc(&x->part_t, 4 * np) != cudaSuccess || cudaMalloc(&x->part_i, 4 * np) != cudaSuccess ||
         cudaMalloc(&x->part_k, 4 * np) != cudaSuccess || cudaMalloc(&x->part_ki, 4 * np) != cudaSuccess)
         return fail(EAD_ECUDA);
+    if (cfg->shard_count > 0) {
+        if (cudaMalloc(&x->link, sizeof(ShardLink)) != cudaSuccess) return fail(EAD_ECUDA);
+        cudaMemsetAsync(x->link, 0, sizeof(ShardLink), x->stream);
+    }
     cudaMemsetAsync(x->ctl, 0, sizeof(StepCtl), x->stream);
     cudaMemsetAsync(x->args, 0, sizeof(RunArgs), x->stream);
     cudaMemsetAsync(x->perm, 0, 8ull * B, x->stream);
@@ -524,19 +562,19 @@ int ead_reset(ead_ctx *x)
 int ead_step(ead_ctx *x, const void *h_small, const void *h_large, int32_t *tok, float *H, float *Hbar,
              uint8_t *model_used, uint8_t *next_model)
 {
-    if (!x || !h_small || !h_large) return EAD_EINVALID_ARG;
+    if (!x || !h_small || !h_large || !can_step(x)) return EAD_EINVALID_ARG;
     if (!aligned16(h_small) || !aligned16(h_large)) return EAD_EALIGNMENT;
     int rc = set_args(x, h_small, h_large, tok, H, Hbar, model_used, next_model, x->stream);
     if (rc != EAD_OK) return rc;
-    rc = enqueue_step(x, x->stream);
-    x->launches += 3;
+    rc = enqueue_step(x, x->stream, nullptr, step_mode(x));
+    x->launches += kernels_per_step(x);
     return rc;
 }
 
 int ead_run(ead_ctx *x, int32_t T, const void *h_small_seq, const void *h_large_seq, int32_t *tok, float *H,
             float *Hbar, uint8_t *model_used, uint8_t *next_model)
 {
-    if (!x || T < 0 || !h_small_seq || !h_large_seq) return EAD_EINVALID_ARG;
+    if (!x || T < 0 || !h_small_seq || !h_large_seq || !can_step(x)) return EAD_EINVALID_ARG;
     if (!aligned16(h_small_seq) || !aligned16(h_large_seq)) return EAD_EALIGNMENT;
     if (T == 0) return EAD_OK;
     return run_device(x, T, h_small_seq, h_large_seq, tok, H, Hbar, model_used, next_model);
@@ -545,7 +583,7 @@ int ead_run(ead_ctx *x, int32_t T, const void *h_small_seq, const void *h_large_
 int ead_run_timed(ead_ctx *x, int32_t T, const void *h_small_seq, const void *h_large_seq, int32_t *tok, float *H,
                   float *Hbar, uint8_t *model_used, uint8_t *next_model, float *kernel_ms)
 {
-    if (!x || T < 0 || !h_small_seq || !h_large_seq || !kernel_ms) return EAD_EINVALID_ARG;
+    if (!x || T < 0 || !h_small_seq || !h_large_seq || !kernel_ms || x->cfg.shard_count > 0) return EAD_EINVALID_ARG;
     if (!aligned16(h_small_seq) || !aligned16(h_large_seq)) return EAD_EALIGNMENT;
     kernel_ms[0] = kernel_ms[1] = kernel_ms[2] = 0.f;
     if (T == 0) return EAD_OK;
@@ -578,7 +616,7 @@ int ead_run_timed(ead_ctx *x, int32_t T, const void *h_small_seq, const void *h_
 int ead_run_host(ead_ctx *x, int32_t T, const void *h_small_seq, const void *h_large_seq, int32_t *tok, float *H,
                  float *Hbar, uint8_t *model_used, uint8_t *next_model)
 {
-    if (!x || T < 0 || !h_small_seq || !h_large_seq) return EAD_EINVALID_ARG;
+    if (!x || T < 0 || !h_small_seq || !h_large_seq || !can_step(x)) return EAD_EINVALID_ARG;
     if (T == 0) return EAD_OK;
     int rc = ensure_staging(x);
     if (rc != EAD_OK) return rc;
@@ -623,6 +661,72 @@ int ead_run_host(ead_ctx *x, int32_t T, const void *h_small_seq, const void *h_l
     return EAD_OK;
 }
 
+int ead_shard_range(int32_t V, int32_t n_shards, int32_t shard, int32_t *begin, int32_t *end)
+{
+    if (V < 1 || n_shards < 1 || shard < 0 || shard >= n_shards || !begin || !end) return EAD_EINVALID_ARG;
+    const int64_t U = (static_cast<int64_t>(V) + kTileM - 1) / kTileM;      // whole 128-row tiles, last one ragged
+    if (n_shards > U) return EAD_EINVALID_ARG;                               // some shard would be empty
+    *begin = static_cast<int32_t>(U * shard / n_shards * kTileM);
+    *end = static_cast<int32_t>(std::min<int64_t>(V, U * (shard + 1) / n_shards * kTileM));
+    return EAD_OK;
+}
+
+size_t ead_shard_exchange_bytes(int32_t B, int32_t n_shards)
+{
+    if (B < 1 || n_shards < 1) return 0;
+    return 2ull * n_shards * B * sizeof(ShardRecord);
+}
+
+int ead_shard_connect(ead_ctx *x, int32_t shard, void *const *exchange)
+{
+    if (!x || !exchange || x->cfg.shard_count < 1 || shard < 0 || shard >= x->cfg.shard_count) return EAD_EINVALID_ARG;
+    ShardLink lk{};
+    lk.n = x->cfg.shard_count;
+    lk.self = shard;
+    for (int d = 0; d < lk.n; ++d) {
+        if (!exchange[d]) return EAD_EINVALID_ARG;
+        if (!aligned16(exchange[d])) return EAD_EALIGNMENT;
+        lk.all[d] = static_cast<ShardRecord *>(exchange[d]);
+    }
+    EAD_CUDA(cudaStreamSynchronize(x->stream));
+    EAD_CUDA(cudaMemcpy(x->link, &lk, sizeof lk, cudaMemcpyHostToDevice));
+    const int32_t zero[2] = {0, 0};                  // record numbering restarts with the fresh buffers
+    EAD_CUDA(cudaMemcpy(&x->ctl->xstep, zero, sizeof zero, cudaMemcpyHostToDevice));
+    x->connected = true;
+    return EAD_OK;
+}
+
+int ead_shard_partials(ead_ctx *x, const void *h_small, const void *h_large, void *records)
+{
+    if (!x || !h_small || !h_large || x->cfg.shard_count < 1 || (!records && !x->connected)) return EAD_EINVALID_ARG;
+    if (!aligned16(h_small) || !aligned16(h_large) || !aligned16(records)) return EAD_EALIGNMENT;
+    int rc = set_args(x, h_small, h_large, nullptr, nullptr, nullptr, nullptr, nullptr, x->stream,
+                      static_cast<float *>(records));
+    if (rc != EAD_OK) return rc;
+    rc = enqueue_step(x, x->stream, nullptr, records ? 1 : 3);
+    x->launches += 3;
+    return rc;
+}
+
+int ead_shard_gate(ead_ctx *x, const void *all_records, int32_t n_shards, int32_t *tok, float *H, float *Hbar,
+                   uint8_t *model_used, uint8_t *next_model)
+{
+    if (!x || x->cfg.shard_count < 1 || n_shards != x->cfg.shard_count || (!all_records && !x->connected))
+        return EAD_EINVALID_ARG;
+    if (!aligned16(all_records)) return EAD_EALIGNMENT;
+    RunArgs out{};
+    out.tok = tok;
+    out.H = H;
+    out.Hbar = Hbar;
+    out.used = model_used;
+    out.next = next_model;
+    const GateParams gp = gate_params(x, 0);
+    ead_shard_gate_kernel<<<(x->cfg.B + 127) / 128, 128, 0, x->stream>>>(
+        gp, static_cast<const ShardRecord *>(all_records), n_shards, out, all_records ? 1 : 3);
+    x->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? EAD_OK : EAD_ECUDA;
+}
+
 int ead_status(ead_ctx *x, uint32_t *status_word)
 {
     if (!x) return EAD_EINVALID_ARG;
@@ -630,7 +734,8 @@ int ead_status(ead_ctx *x, uint32_t *status_word)
     StepCtl h{};
     EAD_CUDA(cudaMemcpy(&h, x->ctl, sizeof h, cudaMemcpyDeviceToHost));
     if (status_word) *status_word = h.status;
-    return (h.status & (kStatusWaitExpired | kStatusBadCount)) ? EAD_EDEVICE_FAULT : EAD_OK;
+    if (h.status & (kStatusWaitExpired | kStatusBadCount)) return EAD_EDEVICE_FAULT;
+    return (h.status & kStatusShardMismatch) ? EAD_ESTATE : EAD_OK;
 }
 
 size_t ead_state_size(const ead_ctx *x)
@@ -774,7 +879,7 @@ void ead_destroy(ead_ctx *x)
     if (x->g_chunk) cudaGraphExecDestroy(x->g_chunk);
     if (x->cap_stream) cudaStreamDestroy(x->cap_stream);
     void *bufs[] = {x->ctl, x->args, x->flag, x->c, x->nfill, x->perm, x->ring, x->hc[0], x->hc[1],
-                    x->part_m, x->part_s, x->part_t, x->part_i, x->usage, x->part_k, x->part_ki, x->done};
+                    x->part_m, x->part_s, x->part_t, x->part_i, x->usage, x->part_k, x->part_ki, x->done, x->link};
     for (void *b : bufs)
         if (b) cudaFree(b);
     cudaGetLastError();

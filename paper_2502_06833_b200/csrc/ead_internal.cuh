@@ -21,6 +21,7 @@ constexpr float kNegSentinel = -1.0e30f;            // "no logit seen yet"; fini
 constexpr uint32_t kStatusNonFinite = 0x1u;
 constexpr uint32_t kStatusWaitExpired = 0x2u;
 constexpr uint32_t kStatusBadCount = 0x4u;
+constexpr uint32_t kStatusShardMismatch = 0x8u;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // bounded waits give up after 2 s
 
 // Step control block (device resident, one per context).
@@ -30,7 +31,9 @@ struct StepCtl {
     int32_t n[2];       // rows served by the small / large head in this step
     uint32_t status;    // sticky EAD_STATUS_* bits
     int32_t n_done;     // rows whose sequence has ended (served by neither head)
-    int32_t pad[2];
+    int32_t xstep;      // vocabulary-sharded use: steps taken since the exchange buffers were
+                        // connected (ead_reset leaves it alone); numbers the exchanged records
+    int32_t cur_x;      // copy of `xstep` taken by the compaction kernel for this step
 };
 
 // Caller buffers of the current ead_step / ead_run call (device resident so that a
@@ -43,9 +46,31 @@ struct RunArgs {
     float *Hbar;
     uint8_t *used;
     uint8_t *next;
+    float *shard_out;   // vocabulary-sharded use: receives this shard's record per row instead
     int32_t run_base;
     int32_t pad;
 };
+
+// Record that one vocabulary shard produces per sequence (caller's row order): the statistics of
+// its slice of the active model's logits, with vocabulary indices of the full head.
+struct ShardRecord {
+    float m, s, t;
+    int32_t idx;
+    float k;            // sampling: largest perturbed logit of the slice ...
+    int32_t ki;         // ... and its index
+    int32_t model;      // head the slice belongs to (must agree between the shards)
+    int32_t step1;      // 1 + number of the exchange step the record belongs to; written last
+};
+
+// Where a shard delivers its records when the exchange runs inside the kernels: all[d] is the
+// exchange buffer of shard d ([2][n][B] records: step parity, source shard, row) as addressable
+// from this GPU; all[self] is local memory.
+constexpr int kMaxShards = 16;
+struct ShardLink {
+    ShardRecord *all[kMaxShards];
+    int32_t n, self;
+};
+static_assert(sizeof(ShardRecord) == 32, "two 16-byte words per record");
 
 // How the CTAs of the LM-head kernel divide one head.  With n rows on the head there
 // are R = ceil(n / 128) row blocks; the first g * R CTAs (g = G / R) form R groups of
@@ -160,6 +185,7 @@ struct LmheadParams {
     float *part_k;         // largest perturbed value
     int32_t *part_ki;      // its column
     const int32_t *perm;   // compacted row -> caller's row (the random stream is per caller row)
+    uint32_t ctr_off[2];   // vocabulary-sharded use: first row of this slice in the full head, / 4
 };
 
 }  // namespace ead

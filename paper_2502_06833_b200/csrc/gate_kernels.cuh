@@ -97,6 +97,7 @@ ead_compact_kernel(StepCtl *ctl, const RunArgs *args, const uint8_t *flag, const
         ctl->n[1] = total_large;
         ctl->n_done = total_done;
         ctl->cur_t = step;
+        ctl->cur_x = ctl->xstep;
     }
     __syncthreads();
 
@@ -141,7 +142,25 @@ struct GateParams {
     uint32_t *usage;           // [3][B]: tokens by the small model, by the large model, switches
     uint8_t *done;             // [B]: the sequence has produced the end-of-sequence token
     int32_t eos_token;         // < 0: none
+    // vocabulary-sharded use: the merge kernels stop after the cross-CTA merge and hand on one
+    // ShardRecord per row (indices shifted by v_off of the row's head): reduce_only = 1 writes
+    // it to args->shard_out (the caller exchanges), 2 stores it into the exchange buffer of
+    // every shard named in `link` (peer memory)
+    int32_t reduce_only;
+    int32_t v_off[2];
+    const ShardLink *link;
 };
+
+__device__ __forceinline__ uint32_t ld_acquire_sys(const int32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_sys(int32_t *p, int32_t v)
+{
+    asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 
 // Everything after the merge for one compacted row (executed by one thread): Eq. 2 in the
 // fused form, then the tail of Algorithm 1's loop body (window, counter, Eq. 4), state update
@@ -168,8 +187,37 @@ __device__ __forceinline__ RowState load_row_state(const GateParams &p, int m, i
 }
 
 __device__ __forceinline__ void finish_row(const GateParams &p, const RowState &st, const Partial &acc, int t_step,
-                                           const Draw &draw)
+                                           const Draw &draw, const RunArgs &out)
 {
+    if (p.reduce_only) {                          // one vocabulary shard: hand the slice's statistics on
+        const int off = p.v_off[st.model];
+        const int step1 = p.ctl->cur_x + 1;
+        const float4 lo = make_float4(acc.m, acc.s, acc.t,
+                                      __int_as_float(acc.idx == 0x7fffffff ? acc.idx : acc.idx + off));
+        const float2 hi = make_float2(draw.k, __int_as_float(draw.ki == 0x7fffffff ? draw.ki : draw.ki + off));
+        if (p.reduce_only == 1) {
+            ShardRecord *dst = reinterpret_cast<ShardRecord *>(out.shard_out) + st.b;
+            *reinterpret_cast<float4 *>(dst) = lo;
+            *reinterpret_cast<float2 *>(&dst->k) = hi;
+            dst->model = st.model;
+            dst->step1 = step1;
+            return;
+        }
+        // Exchange inside the kernel: the record goes straight into every shard's buffer (plain
+        // stores, over NVLink for the peers); the step word follows with release semantics, so a
+        // reader that sees it sees the record.  Buffers alternate with the step's parity: a shard
+        // can be at most one step ahead of another (its next gate needs that shard's next record).
+        const ShardLink &lk = *p.link;
+        const size_t slot = (static_cast<size_t>((step1 - 1) & 1) * lk.n + lk.self) * p.B + st.b;
+        for (int d = 0; d < lk.n; ++d) {
+            ShardRecord *dst = lk.all[d] + slot;
+            *reinterpret_cast<float4 *>(dst) = lo;
+            *reinterpret_cast<float2 *>(&dst->k) = hi;
+            dst->model = st.model;
+        }
+        for (int d = 0; d < lk.n; ++d) st_release_sys(&(lk.all[d] + slot)->step1, step1);
+        return;
+    }
     // ---- Eq. 2 in the fused form  H = ln Z - E_p[z] = ln s - t / (s log2 e)   (nats)
     float H = logf(acc.s) - acc.t / (acc.s * kLog2e);
     const bool finite = isfinite(H) && acc.s > 0.f;
@@ -182,11 +230,11 @@ __device__ __forceinline__ void finish_row(const GateParams &p, const RowState &
     if (!finite) {
         // non-finite logits: report, leave window, counter and model untouched
         atomicOr(&p.ctl->status, kStatusNonFinite);
-        if (p.args->tok) p.args->tok[o] = -1;
-        if (p.args->H) p.args->H[o] = __int_as_float(0x7fc00000);
-        if (p.args->Hbar) p.args->Hbar[o] = __int_as_float(0x7fc00000);
-        if (p.args->used) p.args->used[o] = static_cast<uint8_t>(model);
-        if (p.args->next) p.args->next[o] = static_cast<uint8_t>(model);
+        if (out.tok) out.tok[o] = -1;
+        if (out.H) out.H[o] = __int_as_float(0x7fc00000);
+        if (out.Hbar) out.Hbar[o] = __int_as_float(0x7fc00000);
+        if (out.used) out.used[o] = static_cast<uint8_t>(model);
+        if (out.next) out.next[o] = static_cast<uint8_t>(model);
         return;
     }
     // ---- Algorithm 1: append H_t to W; mean of the last w entries (those present)
@@ -212,11 +260,11 @@ __device__ __forceinline__ void finish_row(const GateParams &p, const RowState &
     if (model != used) p.usage[2 * p.B + b] += 1u;
     const int token = p.sampling ? draw.ki : acc.idx;
     if (p.eos_token >= 0 && token == p.eos_token) p.done[b] = 1;    // "while not done" ends for this row
-    if (p.args->tok) p.args->tok[o] = token;
-    if (p.args->H) p.args->H[o] = H;
-    if (p.args->Hbar) p.args->Hbar[o] = Hbar;
-    if (p.args->used) p.args->used[o] = static_cast<uint8_t>(used);
-    if (p.args->next) p.args->next[o] = static_cast<uint8_t>(model);
+    if (out.tok) out.tok[o] = token;
+    if (out.H) out.H[o] = H;
+    if (out.Hbar) out.Hbar[o] = Hbar;
+    if (out.used) out.used[o] = static_cast<uint8_t>(used);
+    if (out.next) out.next[o] = static_cast<uint8_t>(model);
 }
 
 __device__ __forceinline__ Draw warp_merge_draw(Draw d)
@@ -257,7 +305,7 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const Gate
     const int nd = p.ctl->n_done;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         if (n0 + n1 + nd != p.B) atomicOr(&p.ctl->status, kStatusBadCount);
-        p.ctl->step = t_step + 1;                 // nobody in this kernel reads `step`
+        if (!p.reduce_only) p.ctl->step = t_step + 1;   // nobody in this kernel reads `step`
     }
     if (i >= n0 + n1 || n0 + n1 + nd != p.B) return;
     const int m = i < n0 ? 0 : 1;
@@ -279,7 +327,7 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const Gate
     }
     acc = warp_merge(acc);
     if (p.sampling) draw = warp_merge_draw(draw);
-    if (lane == 0) finish_row(p, load_row_state(p, m, r), acc, t_step, draw);
+    if (lane == 0) finish_row(p, load_row_state(p, m, r), acc, t_step, draw, *p.args);
 }
 
 // One block per compacted row: the 4 G partials of the small-batch kernel.  Thread t folds slots t, t + 256, ... in ascending order, then lanes, then warps:
@@ -313,7 +361,7 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_wide_kernel(const
     griddep_wait();                              // partials of the LM-head kernel
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         if (n0 + n1 + nd != p.B) atomicOr(&p.ctl->status, kStatusBadCount);
-        p.ctl->step = t_step + 1;
+        if (!p.reduce_only) p.ctl->step = t_step + 1;
     }
     if (!live) return;
     const size_t base = (static_cast<size_t>(m) * p.B + r) * p.slots_stride;
@@ -339,8 +387,89 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_wide_kernel(const
             acc = merge_partial(acc, wsum[k]);
             draw = merge_draw(draw, dsum[k]);
         }
-        finish_row(p, st, acc, t_step, draw);
+        finish_row(p, st, acc, t_step, draw, *p.args);
     }
+}
+
+// Vocabulary-sharded use, the step's second half.  One thread per sequence folds the records of
+// all n shards for this step in shard order and finishes the step exactly as the single-GPU
+// merge does.  Every shard runs this on the same records in the same order, so the per-sequence
+// state stays identical on all of them without further communication.
+//   mode 1: `all` = [n][B] records gathered by the caller; outputs `out` are [B]
+//   mode 2: records arrive in this shard's exchange buffer (link->all[self]), stored there by
+//           the merge kernels of all shards; the thread waits for each record's step word
+//           (bounded: a shard that never delivers sets EAD_STATUS_WAIT_EXPIRED); outputs go
+//           to the buffers of the current run (p.args)
+//   mode 3: records as in mode 2, outputs as in mode 1 (the two halves of a step called apart)
+__global__ void __launch_bounds__(128)
+ead_shard_gate_kernel(const GateParams p, const ShardRecord *all, int n_shards, RunArgs out, int mode)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    griddep_launch_dependents();
+    griddep_wait();                               // this shard's own records, state of the last step
+    const int t_step = p.ctl->cur_t;
+    const int step1 = p.ctl->cur_x + 1;
+    if (mode >= 2) {
+        const ShardLink &lk = *p.link;
+        n_shards = lk.n;
+        all = lk.all[lk.self] + static_cast<size_t>((step1 - 1) & 1) * lk.n * p.B;
+    }
+    if (mode == 2) out = *p.args;
+    else out.run_base = t_step;
+    if (b == 0) {                                 // nobody in this kernel reads step or xstep
+        p.ctl->step = t_step + 1;
+        p.ctl->xstep = step1;
+    }
+    if (b >= p.B) return;
+    const int model = p.flag[b];
+    const size_t o = static_cast<size_t>(t_step - out.run_base) * p.B + b;
+    if (p.done[b]) {                              // ended sequence: as the compaction kernel reports it
+        const float nan = __int_as_float(0x7fc00000);
+        if (out.tok) out.tok[o] = -1;
+        if (out.H) out.H[o] = nan;
+        if (out.Hbar) out.Hbar[o] = nan;
+        if (out.used) out.used[o] = static_cast<uint8_t>(model);
+        if (out.next) out.next[o] = static_cast<uint8_t>(model);
+        return;
+    }
+    Partial acc{kNegSentinel, 0.f, 0.f, 0x7fffffff};
+    Draw draw{-INFINITY, 0x7fffffff};
+    bool agree = true;
+    // one deadline for all of this thread's waits; none at all once a wait has expired before
+    bool patient = mode >= 2 && !(p.ctl->status & kStatusWaitExpired);
+    const unsigned long long t0 = patient ? globaltimer_ns() : 0ull;
+    for (int s = 0; s < n_shards; ++s) {
+        const ShardRecord *rec = all + static_cast<size_t>(s) * p.B + b;
+        int got = static_cast<int>(ld_acquire_sys(&rec->step1));
+        while (got != step1 && patient) {
+            __nanosleep(64);
+            got = static_cast<int>(ld_acquire_sys(&rec->step1));
+            if (got != step1 && globaltimer_ns() - t0 > kWaitLimitNs) {
+                atomicOr(&p.ctl->status, kStatusWaitExpired);
+                patient = false;
+            }
+        }
+        // ordinary loads: the acquire above orders them after the writer's release of the step word
+        const float4 lo = *reinterpret_cast<const float4 *>(rec);
+        const float2 hi = *reinterpret_cast<const float2 *>(&rec->k);
+        const int rmodel = rec->model;
+        agree = agree && got == step1 && rmodel == model;
+        acc = merge_partial(acc, Partial{lo.x, lo.y, lo.z, __float_as_int(lo.w)});
+        draw = merge_draw(draw, Draw{hi.x, __float_as_int(hi.y)});
+    }
+    if (!agree) {                                 // a shard is on another step or saw other flags
+        atomicOr(&p.ctl->status, kStatusShardMismatch);
+        acc.s = 0.f;                              // reported like a non-finite row: state untouched
+    }
+    RowState st;
+    st.b = b;
+    st.model = model;
+    st.nf = p.nfill[b];
+    st.c = p.c[b];
+    st.run_base = out.run_base;
+    st.ring_global = p.ring + static_cast<size_t>(b) * p.w;
+    st.ring = st.ring_global;
+    finish_row(p, st, acc, t_step, draw, out);
 }
 
 }  // namespace ead

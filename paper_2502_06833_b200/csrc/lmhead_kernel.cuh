@@ -128,11 +128,12 @@ __device__ __forceinline__ void rowstat_absorb32(RowStat &st, const float (&v)[3
 // Temperature sampling: folds 32 consecutive logits (columns cb .., cb a multiple of 16) of the
 // sequence with random-stream coordinates (step, row) into its running draw.
 __device__ __forceinline__ void draw_absorb32(Draw &dr, const float (&v)[32], int cb, uint32_t rng_step,
-                                              uint32_t rng_row, const LmheadParams &p)
+                                              uint32_t rng_row, const LmheadParams &p, uint32_t ctr_off)
 {
 #pragma unroll
     for (int j = 0; j < 32; j += 4) {
-        const uint4 w = philox4x32_10(static_cast<uint32_t>(cb + j) >> 2, rng_step, rng_row, 0u, p.seed_lo, p.seed_hi);
+        const uint4 w = philox4x32_10((static_cast<uint32_t>(cb + j) >> 2) + ctr_off, rng_step, rng_row, 0u, p.seed_lo,
+                                       p.seed_hi);
         const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -326,7 +327,7 @@ ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
                             for (int j = 0; j < 32; ++j) v[j] = (cb + j < col_limit) ? v[j] : kNegSentinel;
                         }
                         rowstat_absorb32(st, v, cb);
-                        if (SAMPLE && sampling) draw_absorb32(dr, v, cb, rng_step, rng_row, p);
+                        if (SAMPLE && sampling) draw_absorb32(dr, v, cb, rng_step, rng_row, p, p.ctr_off[m]);
                         __syncwarp();
                     }
                 }

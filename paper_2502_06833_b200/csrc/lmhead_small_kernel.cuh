@@ -247,7 +247,7 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                                 for (int i = 0; i < 32; ++i) w[i] = (cb + i < limit) ? w[i] : kNegSentinel;
                             }
                             rowstat_absorb32(st3[ch], w, cb);
-                            if (SAMPLE) draw_absorb32(dr3[ch], w, cb, rng_step, rr3[ch], p);
+                            if (SAMPLE) draw_absorb32(dr3[ch], w, cb, rng_step, rr3[ch], p, p.ctr_off[m]);
                             __syncwarp();
                         }
                     }
@@ -323,7 +323,7 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                     if (SAMPLE) {
 #pragma unroll
                         for (int j = 0; j < NB; ++j) {
-                            const uint4 w = philox4x32_10(static_cast<uint32_t>(row) >> 2, rng_step, rng_row[j], 0u,
+                            const uint4 w = philox4x32_10((static_cast<uint32_t>(row) >> 2) + p.ctr_off[m], rng_step, rng_row[j], 0u,
                                                           p.seed_lo, p.seed_hi);
                             const uint32_t word = (row & 3) == 0 ? w.x : (row & 3) == 1 ? w.y : (row & 3) == 2 ? w.z : w.w;
                             const float key = fmaf(v[j], p.inv_temperature, gumbel_from_word(word));

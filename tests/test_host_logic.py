@@ -152,3 +152,109 @@ def test_parameter_ratio_matches_the_table_footnote(E):
     assert 100 * E.ead_parameter_ratio(84, 16, 1, 3) == pytest.approx(44.0, abs=0.05)
     assert E.ead_parameter_ratio(10, 0, 3, 11) == pytest.approx(3 / 11)
     assert E.ead_parameter_ratio(0, 10, 3, 11) == 1.0
+
+
+def test_shard_ranges_cover_the_vocabulary_in_whole_tiles(E):
+    for V, n in [(128256, 8), (152064, 4), (1100, 2), (1024, 8), (129, 2), (5, 1)]:
+        cuts = [E.ead_shard_range(V, n, r) for r in range(n)]
+        assert cuts[0][0] == 0 and cuts[-1][1] == V
+        for (b0, e0), (b1, _) in zip(cuts, cuts[1:]):
+            assert e0 == b1
+        for b, e in cuts:
+            assert b % 128 == 0 and e > b
+        tiles = [-(-(e - b) // 128) for b, e in cuts]
+        assert max(tiles) - min(tiles) <= 1                       # dealt out evenly
+    with pytest.raises(E.EadError) as err:                        # 9 tiles cannot feed 10 shards
+        E.ead_shard_range(1100, 10, 0)
+    assert err.value.code == E.EAD_EINVALID_ARG
+    with pytest.raises(E.EadError):
+        E.ead_shard_range(1100, 2, 2)
+
+
+# Two gloo ranks drive VocabParallelGate with a numpy stand-in for the CUDA library (same call
+# names and record layout).  What is under test is the glue: slice bounds, the order of the
+# gathered records, and that merging per-slice statistics in rank order gives the
+# full-vocabulary entropy and arg max of the oracle.
+_VP_WORKER = r"""
+import os, sys
+sys.path.insert(0, {root!r})
+sys.path.insert(0, os.path.join({root!r}, "tests"))
+import numpy as np, torch, torch.distributed as dist
+from paper_2502_06833_b200 import binding, vocab_parallel as VP
+from oracle import ead_oracle as O
+
+LOG2E = 1.4426950408889634
+
+class FakeEngine:
+    EAD_SHARD_RECORD_BYTES = 32
+    ead_shard_range = staticmethod(binding.ead_shard_range)
+    def ead_create(self, **kw):
+        self.kw = kw
+        self.step = 0
+        return self
+    def ead_shard_partials(self, ctx, h_small, h_large, records):
+        W, off = self.kw["W_small"].double().numpy(), self.kw["vocab_offset_small"]   # every row starts on M_S
+        z = h_small.double().numpy() @ W.T                                              # [B, slice]
+        m = z.max(1)
+        e = np.exp(z - m[:, None])
+        rec = records.numpy()
+        rec[:, 0], rec[:, 1], rec[:, 2] = m, e.sum(1), (e * (z - m[:, None])).sum(1) * LOG2E
+        ints = rec.view(np.int32)
+        ints[:, 3] = z.argmax(1) + off
+        ints[:, 6], ints[:, 7] = 0, self.step
+    def ead_shard_gate(self, ctx, all_records, n, tok, H, Hbar, used, nxt):
+        a = all_records.numpy().astype(np.float64)
+        ai = all_records.numpy().view(np.int32)
+        assert n == self.kw["shard_count"] and (ai[:, :, 7] == self.step).all()
+        B = a.shape[1]
+        for b in range(B):
+            m, s, t, idx = -1e30, 0.0, 0.0, 2**31 - 1
+            for r in range(n):
+                qm, qs, qt, qi = a[r, b, 0], a[r, b, 1], a[r, b, 2], int(ai[r, b, 3])
+                M = max(m, qm)
+                da, db = (m - M) * LOG2E, (qm - M) * LOG2E
+                ea, eb = 2.0 ** da, 2.0 ** db
+                s, t = ea * s + eb * qs, ea * (da * s + t) + eb * (db * qs + qt)
+                idx = idx if m > qm else qi if qm > m else min(idx, qi)
+                m = M
+            H[b] = np.log(s) - t / (s * LOG2E)
+            tok[b] = idx
+        self.step += 1
+    def ead_destroy(self, ctx): pass
+
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+rng = np.random.default_rng(5)
+V, Hd, B = 1100, 32, 3
+W = torch.from_numpy(rng.integers(-24, 25, (V, Hd)) / 16.0).float()          # exact in bf16 and float32
+h = torch.from_numpy(rng.integers(-16, 17, (B, Hd)) / 8.0).float()
+Wl = torch.zeros((V, 8))
+gate = VP.VocabParallelGate(B=B, V_small=V, V_large=V, H_small=Hd, H_large=8, w=5, d_min=10, tau=1.0,
+                            W_small=VP.shard_of(W, world, rank), W_large=VP.shard_of(Wl, world, rank),
+                            rank=rank, world=world, engine=FakeEngine(), device=torch.device("cpu"))
+assert gate.W_small.shape[0] == (512 if rank == 0 else 588)        # 9 tiles: 4 + 5 (ragged)
+tok = torch.zeros(B, dtype=torch.int32); H = torch.zeros(B, dtype=torch.float32)
+gate.step(h, torch.zeros((B, 8)), tok, H)
+# records arrived in rank order: slice r's arg max lies in slice r
+ints = gate.all_records.numpy().view(np.int32)
+for r in range(world):
+    b, e = VP.shard_rows(V, world, r)
+    assert ((ints[r, :, 3] >= b) & (ints[r, :, 3] < e)).all()
+z = h.double().numpy() @ W.double().numpy().T
+for b in range(B):
+    assert abs(float(H[b]) - O.entropy(z[b])) < 1e-6, (float(H[b]), O.entropy(z[b]))
+    assert int(tok[b]) == O.greedy(z[b])[0]
+dist.barrier()
+dist.destroy_process_group()
+print("rank", rank, "ok")
+"""
+
+
+def test_vocab_parallel_glue_over_two_gloo_ranks(tmp_path):
+    script = tmp_path / "vp_worker.py"
+    script.write_text(_VP_WORKER.format(root=ROOT))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+           "--master-addr", "127.0.0.1", "--master-port", "29633", str(script)]
+    res = subprocess.run(cmd, capture_output=True, text=True, timeout=240)
+    assert res.returncode == 0, res.stdout + res.stderr
+    assert res.stdout.count("ok") == 2
