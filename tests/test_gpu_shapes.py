@@ -201,6 +201,30 @@ def test_largest_batch_and_zero_steps():
     compare(out, ora, cfg.tau)
 
 
+def test_maximum_batch_of_the_interface():
+    """B = 4096, the largest batch ead_create takes: 32 row blocks over both heads, four or
+    five CTAs per row block."""
+    cfg = _cfg(B=4096, V=700, H_small=16, H_large=8, T=3, tau=_mid_tau(700), d_min=1, w=2)
+    wl = synth.Workload(cfg)
+    ora = _oracle(cfg, wl)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        out = g.run(wl.h_small, wl.h_large, "run")
+    compare(out, ora, cfg.tau)
+    assert 0 < ora["used"].mean() < 1
+
+
+def test_vocabulary_of_thousands_of_tiles():
+    """A vocabulary twice the size of the largest configuration's (narrow heads keep it cheap):
+    every CTA walks many tiles, the last one ragged."""
+    cfg = _cfg(B=2, V=300007, H_small=8, H_large=16, T=3, tau=_mid_tau(300007), d_min=1)
+    wl = synth.Workload(cfg)
+    ora = _oracle(cfg, wl)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        out = g.run(wl.h_small, wl.h_large, "run")
+    compare(out, ora, cfg.tau)
+    assert out["tok"].max() > 2 ** 17
+
+
 def test_usage_counters_follow_the_trace_and_survive_a_checkpoint():
     cfg = _cfg(B=6, V=1500, T=40, tau=_mid_tau(1500))
     wl = synth.Workload(cfg)
