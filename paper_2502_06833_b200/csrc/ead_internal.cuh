@@ -186,6 +186,7 @@ struct LmheadParams {
     int32_t *part_ki;      // its column
     const int32_t *perm;   // compacted row -> caller's row (the random stream is per caller row)
     uint32_t ctr_off[2];   // vocabulary-sharded use: first row of this slice in the full head, / 4
+    int32_t prefetch_boxes;  // small-batch kernel: 16 KiB weight boxes brought into L2 before the dependency wait
 };
 
 }  // namespace ead

@@ -94,9 +94,6 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&ctrl->tmem_base);
-    // Everything above touched no global memory: it may overlap the kernels before this one.
-    griddep_wait();
-    griddep_launch_dependents();
     const int cta = blockIdx.x;
     int row_begin_m[2], row_end_m[2];            // this CTA's vocabulary range on each head
 #pragma unroll
@@ -105,6 +102,25 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
         row_begin_m[m] = static_cast<int>(n_seg * cta / G) * kSmallSegRows;
         row_end_m[m] = static_cast<int>(n_seg * (cta + 1) / G) * kSmallSegRows;
     }
+    // Everything above touched no global memory: it may overlap the kernels before this one.
+    // So may this: while the previous step's merge and this step's compaction run, HBM is idle.
+    // The weights do not depend on them, so the first boxes of this CTA's range are brought
+    // into L2 now, for the head that served rows in the previous step (a guess from a counter
+    // that the compaction kernel may be rewriting: a wrong guess costs bandwidth, nothing else).
+    if (warp == 0 && lane == 0 && p.prefetch_boxes > 0) {
+        const int g0 = *reinterpret_cast<const volatile int32_t *>(&p.ctl->n[0]);
+        const int g1 = *reinterpret_cast<const volatile int32_t *>(&p.ctl->n[1]);
+        const int m = g0 > 0 ? 0 : 1;
+        if (g0 > 0 || g1 > 0) {
+            const CUtensorMap *tW = m ? &tmW1 : &tmW0;
+            const int kcols = (p.H[m] + 63) / 64;
+            int left = p.prefetch_boxes;
+            for (int row0 = row_begin_m[m]; row0 < row_end_m[m] && left > 0; row0 += kSmallTileRows)
+                for (int kc = 0; kc < kcols && left > 0; ++kc, --left) tma_prefetch_l2_2d(tW, kc * 64, row0);
+        }
+    }
+    griddep_wait();
+    griddep_launch_dependents();
     const int n_rows[2] = {p.ctl->n[0], p.ctl->n[1]};
 
     if (warp == 0) {

@@ -81,6 +81,15 @@ __device__ __forceinline__ void tma_prefetch_desc(const void *tmap)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
 }
+// Brings the box at (x, y) of a 2-D tiled tensor into L2 only (no shared-memory destination, no
+// completion to wait for).  Same alignment rule for x as a load.
+__device__ __forceinline__ void tma_prefetch_l2_2d(const void *tmap, int32_t x, int32_t y)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(
+                     reinterpret_cast<uint64_t>(tmap)),
+                 "r"(x), "r"(y)
+                 : "memory");
+}
 // 2-D tiled load global -> shared, completion counted in bytes on an mbarrier.
 // x is the innermost (contiguous) coordinate in elements and must make
 // x * sizeof(element) a multiple of 16.

@@ -216,10 +216,10 @@ def test_whole_runs_through_the_exchange_buffer_of_a_single_shard(B, V):
         g.run(cfg.T, hs, hl, o["tok"], o["H"], o["Hbar"], o["used"], o["next"])
         g.status()
         first = {k: v.cpu().numpy() for k, v in o.items()}
-        g.reset()                                                    # record numbering carries on: odd step count so far? 70 is even
+        g.reset()                                                    # the numbering of exchanged records carries on
         o2 = sh._outs(7)
         g.run(7, hs, hl, o2["tok"], o2["H"], o2["Hbar"], o2["used"], o2["next"])
-        g.reset()                                                    # 77 exchange steps taken: parity differs from step 0's
+        g.reset()                                                    # 77 exchanges so far: step 0 now lands in the other buffer
         o3 = sh._outs(cfg.T)
         for t in range(cfg.T):                                       # step by step through ead_step
             g.step(hs[t], hl[t], o3["tok"][t], o3["H"][t], o3["Hbar"][t], o3["used"][t], o3["next"][t])
