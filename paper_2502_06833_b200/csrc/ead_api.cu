@@ -23,7 +23,7 @@ namespace {
 
 constexpr int kMidCols = 32;              // value of ead_ctx::small_cols that selects ead_lmhead_small_kernel<0>
 #ifndef EAD_PREFETCH_BOXES
-#define EAD_PREFETCH_BOXES 24
+#define EAD_PREFETCH_BOXES 32
 #endif
 constexpr int kPrefetchBoxes = EAD_PREFETCH_BOXES;   // 16 KiB weight boxes per CTA fetched into L2 ahead of the dependency wait
 constexpr int kGraphChunk = 32;           // gate steps unrolled in the replayed graph
