@@ -6,6 +6,7 @@ kernel ever waits for another.  What must hold: every shard ends each step with 
 outputs, bit for bit, and those outputs are the oracle's full-vocabulary results.
 """
 import math
+import time
 
 import numpy as np
 import pytest
@@ -180,6 +181,55 @@ def test_records_from_another_step_are_refused():
         after = E.ead_get_state(g.ctx)
         # windows, counters and flags are those of before the step; only the step count moved on
         assert bytes(before)[16:] == bytes(after)[16:]
+
+
+def test_a_shard_that_never_delivers_ends_the_wait_with_a_status():
+    """Failure detection without a fault: shard 1 stays silent, so the step word that shard 0's
+    gate polls is never set.  Its wait must give up after its limit (2 s), report
+    EAD_STATUS_WAIT_EXPIRED, leave the per-sequence state alone, and the context must stay
+    usable: after a reset and a fresh connect both shards run the workload to the oracle's
+    results."""
+    cfg = _cfg(B=3, V=1000, T=12, tau=_mid_tau(1000))
+    wl = synth.Workload(cfg)
+    ora = O.run(wl.W_small, wl.W_large, wl.h_small, wl.h_large, w=cfg.w, d_min=cfg.d_min,
+                tau=float(np.float32(cfg.tau)))
+    with Shards(cfg, wl.W_small, wl.W_large, 2, peer=True) as sh:
+        E, torch = sh.E, sh.torch
+        g0 = sh.gates[0]
+        hs, hl = to_dev_bf16(wl.h_small), to_dev_bf16(wl.h_large)
+        before = E.ead_get_state(g0.ctx)
+        H = torch.zeros(cfg.B, dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        t0 = time.time()
+        E.ead_shard_partials(g0.ctx, hs[0], hl[0], None)             # shard 0 delivers to both buffers
+        E.ead_shard_gate(g0.ctx, None, 2, None, H, None, None, None)  # ... and waits for shard 1 in vain
+        word = E.ead_status(g0.ctx, raise_on_fault=False)
+        waited = time.time() - t0
+        assert word & E.EAD_STATUS_WAIT_EXPIRED
+        with pytest.raises(E.EadError) as err:
+            E.ead_status(g0.ctx)
+        assert err.value.code == E.EAD_EDEVICE_FAULT
+        assert 1.5 < waited < 20.0, waited
+        assert np.isnan(H.cpu().numpy()).all()                       # reported like a row without a result
+        after = E.ead_get_state(g0.ctx)
+        assert bytes(before)[16:] == bytes(after)[16:]               # windows, counters, flags untouched
+        # a second wait on the same context does not stall again: the expiry is sticky
+        t1 = time.time()
+        E.ead_shard_partials(g0.ctx, hs[0], hl[0], None)
+        E.ead_shard_gate(g0.ctx, None, 2, None, H, None, None, None)
+        E.ead_status(g0.ctx, raise_on_fault=False)
+        assert time.time() - t1 < 1.0
+        # recovery: clear the state and the status, renumber the exchange, run for real
+        torch.cuda.synchronize()
+        for x in sh.exchange:
+            x.zero_()                                                # connect expects fresh buffers
+        for g in sh.gates:
+            g.reset()
+            g.connect(sh.exchange)
+        assert E.ead_status(g0.ctx) == 0
+        outs = sh.run(wl.h_small, wl.h_large)
+    _same_on_all_shards(outs)
+    compare(outs[0], ora, cfg.tau)
 
 
 def test_plain_calls_are_refused_on_a_sharded_context_and_vice_versa():
