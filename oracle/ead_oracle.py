@@ -35,7 +35,9 @@ def _p(a, ctype):
 def lib():
     global _lib
     if _lib is None:
-        L = C.CDLL(build())
+        # EAD_ORACLE_LIB: another build of this file's C source, for the test that plants
+        # mistakes in copies of the oracle and checks that the pins notice
+        L = C.CDLL(os.environ.get("EAD_ORACLE_LIB") or build())
         L.oracle_entropy.restype = C.c_double
         L.oracle_entropy.argtypes = [C.POINTER(C.c_double), C.c_int64, C.c_int,
                                      C.POINTER(C.c_double)]
