@@ -443,14 +443,14 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
         x->small_cols = 1;
         while (x->small_cols < cfg->B) x->small_cols *= 2;
         x->a_rows = cfg->B <= 8 ? 8 : kSmallN;
-        stage_bytes = small_stage_bytes(x->a_rows);
+        stage_bytes = small_stage_bytes(x->a_rows, small_slabs(1));
         x->small_slots = x->G * kSmallSlotsPerCta;
         x->slots_stride = (x->small_slots + 31) & ~31;
     } else if (cfg->B <= kMidMaxRows) {
         // still bound by streaming the weights: same kernel, sequences in chunks of 32
         x->small_cols = kMidCols;
         x->a_rows = (cfg->B + 15) / 16 * 16;
-        stage_bytes = small_stage_bytes(x->a_rows);
+        stage_bytes = small_stage_bytes(x->a_rows, small_slabs(0));
         x->small_slots = x->G * kSmallSlotsPerCta;
         x->slots_stride = (x->small_slots + 31) & ~31;
     } else {

@@ -19,8 +19,8 @@
 // others are done, so the HBM stays busy; measured cost of the imbalance against dynamic
 // scheduling of 256 KB units: 3-4 %.)
 //
-// Pipeline: per K block of 128 hidden elements one stage = two 64-wide W boxes (<= 128 rows
-// each, 16 KiB) + two 64-wide boxes of the compacted hidden rows (8 rows if B <= 8, else 16;
+// Pipeline: per K block of 256 hidden elements (128 for NB = 0) one stage = four (two) 64-wide W boxes
+// (<= 128 rows each, 16 KiB) + as many 64-wide boxes of the compacted hidden rows (8 rows if B <= 8, else 16;
 // the MMA's N = 16 then reads the following kilobyte as rows 8-15, which only feeds
 // accumulator columns nobody reads).  TMEM holds two 16-column accumulators so that the
 // epilogue overlaps the next tile's MMAs.
@@ -40,10 +40,13 @@ constexpr int kSmallTileRows = 128;                    // vocabulary rows per ti
 constexpr int kSmallSegRows = 32;                      // granularity of a CTA's vocabulary range
 constexpr int kSmallSlotsPerCta = 4;                   // one partial per epilogue warp
 constexpr int kSmallN = 16;                            // batch columns (MMA N)
-constexpr int kSmallBlockK = 128;                      // hidden elements per stage
+// 64-wide K slabs per stage: four for B <= 16 (measured on the LLaMA B = 1 step: 163.9 us against
+// 170.3 with two, the same bytes in flight behind half as many barrier round trips), two for the
+// NB = 0 variant, whose hidden-row boxes are up to 16 KiB per slab
+__host__ __device__ constexpr int small_slabs(int nb) { return nb == 0 ? 2 : 4; }
 constexpr int kSmallWBytes = kSmallTileRows * 64 * 2;  // one 64-wide box of W rows: 16 KiB
 constexpr int kMidMaxRows = 128;                       // largest batch of the NB = 0 variant
-__host__ __device__ constexpr int small_stage_bytes(int h_rows) { return 2 * h_rows * 128 + 2 * kSmallWBytes; }
+__host__ __device__ constexpr int small_stage_bytes(int h_rows, int slabs) { return slabs * (h_rows * 128 + kSmallWBytes); }
 
 template <int NB, bool SAMPLE>
 __global__ void __launch_bounds__(kLmheadThreads, 1)
@@ -63,7 +66,9 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
     const int G = gridDim.x;
     const int stages = p.stages;
     const uint32_t h_slab = static_cast<uint32_t>(p.a_rows) * 128;      // hidden rows of one 64-wide K slab
-    const uint32_t stage_bytes = 2 * h_slab + 2 * kSmallWBytes;
+    constexpr int kSlabs = small_slabs(NB);
+    constexpr int kSmallBlockK = 64 * kSlabs;                           // hidden elements per stage
+    const uint32_t stage_bytes = kSlabs * h_slab + kSlabs * kSmallWBytes;
     constexpr uint32_t kAccCols = NB == 0 ? 128u : static_cast<uint32_t>(kSmallN);   // TMEM columns per accumulator
     float *trans = reinterpret_cast<float *>(stage0 + static_cast<size_t>(stages) * stage_bytes);   // NB = 0 only
     StepCtl *ctl = p.ctl_rw;
@@ -138,7 +143,7 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                 const int kblocks = (p.H[m] + kSmallBlockK - 1) / kSmallBlockK;
                 for (int row0 = row_begin; row0 < row_end && ok; row0 += kSmallTileRows) {
                     const int nrows = min(kSmallTileRows, row_end - row0);        // multiple of 32
-                    const uint32_t tx = 2 * (h_slab + static_cast<uint32_t>(nrows) * 128);
+                    const uint32_t tx = kSlabs * (h_slab + static_cast<uint32_t>(nrows) * 128);
                     for (int kb = 0; kb < kblocks; ++kb, ++it) {
                         const uint32_t s = it % stages;
                         const uint32_t ph = (it / stages) & 1u;
@@ -147,10 +152,10 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                         const uint32_t sa = smem_u32(stage0 + static_cast<size_t>(s) * stage_bytes);
                         mbar_arrive_expect_tx(bar, tx);
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
+                        for (int h = 0; h < kSlabs; ++h) {
                             const int k0 = kb * kSmallBlockK + h * 64;
                             tma_load_2d(sa + h * h_slab, tA, k0, 0, bar, pol_keep);
-                            const uint32_t wdst = sa + 2 * h_slab + h * kSmallWBytes;
+                            const uint32_t wdst = sa + kSlabs * h_slab + h * kSmallWBytes;
                             if (nrows == kSmallTileRows) {
                                 tma_load_2d(wdst, tW, k0, row0, bar, pol_keep);
                             } else {
@@ -196,9 +201,9 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                         tc_fence_after_sync();
                         const uint32_t sa = smem_u32(stage0 + static_cast<size_t>(s) * stage_bytes);
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
+                        for (int h = 0; h < kSlabs; ++h) {
                             const uint64_t dh = umma_smem_desc(sa + h * h_slab);                         // B: hidden rows
-                            const uint64_t dw = umma_smem_desc(sa + 2 * h_slab + h * kSmallWBytes);      // A: W rows
+                            const uint64_t dw = umma_smem_desc(sa + kSlabs * h_slab + h * kSmallWBytes);      // A: W rows
 #pragma unroll
                             for (int k = 0; k < 4; ++k)
                                 umma_bf16(d_tmem, dw + 2 * k, dh + 2 * k, idesc, (kb | h | k) != 0);
