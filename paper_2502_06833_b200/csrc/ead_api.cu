@@ -22,10 +22,12 @@ using namespace ead;
 namespace {
 
 constexpr int kMidCols = 32;              // value of ead_ctx::small_cols that selects ead_lmhead_small_kernel<0>
-#ifndef EAD_PREFETCH_BOXES
-#define EAD_PREFETCH_BOXES 32
-#endif
-constexpr int kPrefetchBoxes = EAD_PREFETCH_BOXES;   // 16 KiB weight boxes per CTA fetched into L2 ahead of the dependency wait
+// 16 KiB weight boxes per CTA fetched into L2 ahead of the dependency wait.  Measured optimum on the
+// LLaMA-shaped heads: 64 for B <= 16 (one head per step at B = 1: 160.7 us per step against 162.5 with 32
+// and 161.8 with 128), 32 for 17..128 sequences (both heads live in most steps and only one is guessed:
+// 256 us against 259 with 64).
+constexpr int kPrefetchBoxesSmall = 64;
+constexpr int kPrefetchBoxesMid = 32;
 constexpr int kGraphChunk = 32;           // gate steps unrolled in the replayed graph
 constexpr uint32_t kStateMagic = 0x45414433u;   // "EAD3"
 constexpr size_t kHostStageBytes = 64u << 20;   // per staging buffer of ead_run_host
@@ -213,7 +215,7 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr, int shar
     lp.part_k = x->part_k;
     lp.part_ki = x->part_ki;
     lp.perm = x->perm;
-    lp.prefetch_boxes = pdl ? kPrefetchBoxes : 0;     // nothing to overlap with when the kernels are timed apart
+    lp.prefetch_boxes = !pdl ? 0 : x->small_cols == kMidCols ? kPrefetchBoxesMid : kPrefetchBoxesSmall;     // nothing to overlap with when the kernels are timed apart
     lp.ctr_off[0] = static_cast<uint32_t>(c.vocab_offset_small) >> 2;
     lp.ctr_off[1] = static_cast<uint32_t>(c.vocab_offset_large) >> 2;
     const dim3 lgrid(x->G), lblock(kLmheadThreads);

@@ -132,6 +132,10 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
         // ------------------------------------------------------------- TMA producer
         if (lane == 0) {
             const uint64_t pol_keep = l2_policy_evict_last();
+            // W is read once per step: streamed lines should leave L2 first, not the hidden rows and
+            // not the boxes that the next step's kernel prefetches while this one drains
+            // (measured: LLaMA B = 1 step 164.4 -> 161.6 us, small head only 88.5 -> 84.2 us)
+            const uint64_t pol_w = l2_policy_evict_first();
             uint32_t it = 0;
             bool ok = true;
             for (int m = 0; m < 2 && ok; ++m) {
@@ -157,10 +161,10 @@ ead_lmhead_small_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_c
                             tma_load_2d(sa + h * h_slab, tA, k0, 0, bar, pol_keep);
                             const uint32_t wdst = sa + kSlabs * h_slab + h * kSmallWBytes;
                             if (nrows == kSmallTileRows) {
-                                tma_load_2d(wdst, tW, k0, row0, bar, pol_keep);
+                                tma_load_2d(wdst, tW, k0, row0, bar, pol_w);
                             } else {
                                 for (int j = 0; j < nrows; j += kSmallSegRows)
-                                    tma_load_2d(wdst + j * 128, tP, k0, row0 + j, bar, pol_keep);
+                                    tma_load_2d(wdst + j * 128, tP, k0, row0 + j, bar, pol_w);
                             }
                         }
                     }
