@@ -38,8 +38,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per LM-head launch from the committed ncu
 # capture of the same kernel (profiles/), keyed by config; None until captured for the
 # kernel as it stands.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama_b1": 1.05726e9, "llama_b64": 1.5823e9, "qwen_b256": 2.0374e9,
-                                "qwen_b1024_f100": 1.5878e9}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama_b1": 1.05726e9, "llama_b1_small_only": 5.3285e8, "llama_b64": 1.5823e9,
+                                "qwen_b256": 2.0374e9, "qwen_b1024_f0": 4.7419e8, "qwen_b1024_f25": 2.0679e9,
+                                "qwen_b1024_f50": 2.0830e9, "qwen_b1024_f100": 1.5878e9}
 
 
 def load_peaks():
