@@ -2,23 +2,35 @@
 """Benchmark of the EAD gate step (one step = compaction, LM-head contraction with the
 fused entropy / arg-max epilogue, merge, window + dwell + threshold update) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME|all] [--repeats R]
+                    [--temperature T] [--impl ours|reference]
 
-Prints ONE JSON line (rank 0).  `value` is gate steps per second over all GPUs with the
-inputs resident in HBM; `e2e` is the same through the host-buffer entry point
-(`ead_run_host`), host<->device copies inside the timed region; `roofline` is the
-LM-head kernel's achieved fraction of the binding bound, its duration measured with CUDA
-events around every launch; `cpu_baseline` is the fp64 CPU oracle timed on a bounded
-sample of the same workload.  With N > 1 every rank runs an independent replica of the
-workload (the path has no cross-sequence term and is not sharded).
+Prints ONE JSON line (rank 0).  The headline workload is the LLaMA-shaped B = 1 latency
+configuration: `value` is gate steps per second over all GPUs with the inputs resident in
+HBM (W warm-up steps, then EXACTLY K timed steps, the timed region repeated R >= 10 times
+from the same checkpointed state, median reported, every repeat listed); `e2e` is the same
+through the host-buffer entry point (`ead_run_host`), host<->device copies inside the timed
+region; `roofline` is the LM-head kernel's achieved fraction of the binding bound, its
+duration measured with CUDA events around every launch; `cpu_baseline` is the fp64 CPU
+oracle timed on a bounded sample of the same workload.
 
-`--impl reference` times the CPU oracle alone (there is no reference implementation of
-this path): rank 0 only, a bounded number of steps.
+Without `--config` (or with `--config all`) the same line carries `per_config`: one entry
+per benchmark configuration (LLaMA-shaped B = 1 on the large head, on the small head and
+switching; B = 64; Qwen-shaped B = 256; B = 1024 with 0 / 25 / 50 / 100 % of the rows on the
+large head; two rows with temperature sampling), each measured by the same protocol with
+at least 32 warm-up steps (so that the mix of heads is the configuration's, not that of
+Algorithm 1's first d_min tokens) and at least 32 timed steps per repeat.  `--config NAME`
+measures that configuration alone.
+
+With N > 1 every rank runs an independent replica of the workload (the path has no
+cross-sequence term and is not sharded).  `--impl reference` times the CPU oracle alone
+(there is no reference implementation of this path): rank 0 only, a bounded number of steps.
 """
 from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import sys
 import threading
@@ -34,13 +46,32 @@ from workloads import configs, synth  # noqa: E402
 
 METRIC = "ead_gate_steps_per_s"
 UNIT = "steps/s"
+HEADLINE = "llama_b1"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per LM-head launch from the committed ncu
-# capture of the same kernel (profiles/), keyed by config; None until captured for the
-# kernel as it stands.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama_b1": 1.05726e9, "llama_b1_small_only": 5.3285e8, "llama_b64": 1.5823e9,
-                                "qwen_b256": 2.0374e9, "qwen_b1024_f0": 4.7419e8, "qwen_b1024_f25": 2.0679e9,
-                                "qwen_b1024_f50": 2.0830e9, "qwen_b1024_f100": 1.5878e9}
+# Configurations of the `per_config` list: (workload, temperature).
+PER_CONFIG = [("llama_b1", 0.0), ("llama_b1_small_only", 0.0), ("llama_b1_switching", 0.0),
+              ("llama_b64", 0.0), ("qwen_b256", 0.0), ("qwen_b1024_f0", 0.0), ("qwen_b1024_f25", 0.0),
+              ("qwen_b1024_f50", 0.0), ("qwen_b1024_f100", 0.0), ("llama_b1", 1.0), ("qwen_b1024_f0", 1.0)]
+PER_CONFIG_MIN_WARMUP = 32
+PER_CONFIG_MIN_STEPS = 32
+MIN_REPEATS = 10
+MAX_REPEATS = 40
+TARGET_TIMED_SECONDS = 0.25          # repeats are added until the timed regions sum to this
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one LM-head launch, from the ncu captures
+# committed under profiles/ (file named beside each figure), keyed by workload and by the
+# heads that served rows in the captured launch.  An entry is None once the kernel it was
+# taken from has changed.  A run reports the figure only for the share of its timed steps
+# with the same live heads; workloads whose steps differ mix the per-head figures.
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    ("llama_b1", "large"): (1.05726e9, "profiles/lmhead_small_kernel_llama_b1_ncu_full.md"),
+    ("llama_b1", "small"): (5.3285e8, "profiles/lmhead_kernels_other_configs_ncu_counters.md"),
+    ("llama_b64", "both"): (1.5823e9, "profiles/lmhead_small_kernel_llama_b64_ncu_full.md"),
+    ("qwen_b256", "both"): None,
+    ("qwen_b1024", "small"): None,
+    ("qwen_b1024", "both"): None,
+    ("qwen_b1024", "large"): None,
+}
 
 
 def load_peaks():
@@ -60,9 +91,9 @@ _REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown"
 
 class ClockSampler:
     """Reads SM clock and clock-event reasons of this process's GPU through NVML (read
-    only) every few milliseconds while the timed region runs."""
+    only) every few milliseconds while the timed regions run."""
 
-    def __init__(self, uuid: str | None, period_s: float = 0.01):
+    def __init__(self, uuid: str | None, period_s: float = 0.004):
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
         self._thread = None
@@ -143,6 +174,54 @@ def aggregate_over_ranks(elapsed_ms: float, steps: int, dist=None):
     return world * steps / (t * 1e-3), t, world
 
 
+def roofline_of(bytes_per_launch: float, flops_per_launch: float, kernel_s: float, step_s: float,
+                peaks: dict) -> dict:
+    """Binding bound of one LM-head launch and the achieved fraction of it.  The bound is the
+    slower of (algorithmic bytes / measured copy rate) and (flops / measured sustained bf16
+    rate); tensor-bound rows also state the fraction of the burst rate."""
+    t_hbm = bytes_per_launch / (peaks["hbm_gbs"] * 1e9)
+    t_mma = flops_per_launch / (peaks["bf16_tflops_sustained"] * 1e12)
+    if t_hbm >= t_mma:
+        r = {"bound": "hbm", "achieved": bytes_per_launch / kernel_s / 1e9, "peak": peaks["hbm_gbs"],
+             "unit": "GB/s"}
+        r["frac"] = r["achieved"] / r["peak"]
+        r["frac_of_burst"] = None
+        r["step_frac"] = bytes_per_launch / step_s / 1e9 / peaks["hbm_gbs"]
+        r["step_frac_of_burst"] = None
+        r["peak_source"] = peaks["source"] + " (copy rate)"
+    else:
+        r = {"bound": "tensor", "achieved": flops_per_launch / kernel_s / 1e12,
+             "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
+        r["frac"] = r["achieved"] / r["peak"]
+        r["frac_of_burst"] = r["achieved"] / peaks["bf16_tflops"]
+        r["step_frac"] = flops_per_launch / step_s / 1e12 / peaks["bf16_tflops_sustained"]
+        r["step_frac_of_burst"] = flops_per_launch / step_s / 1e12 / peaks["bf16_tflops"]
+        r["peak_burst"] = peaks["bf16_tflops"]
+        r["peak_source"] = peaks["source"] + " (sustained bf16; burst beside it)"
+    r["bound_us"] = {"hbm": t_hbm * 1e6, "tensor_sustained": t_mma * 1e6}
+    return r
+
+
+def ncu_traffic(cfg, used: np.ndarray):
+    """DRAM bytes per LM-head launch of this run's mix of steps from the committed ncu
+    captures, or None when no (current) capture covers it."""
+    family = "qwen_b1024" if cfg.name.startswith("qwen_b1024") else \
+        "llama_b1" if cfg.name.startswith("llama_b1") else cfg.name
+    n_large = used.sum(axis=1)
+    kinds = np.where(n_large == 0, 0, np.where(n_large == cfg.B, 2, 1))     # small / both / large
+    total, files = 0.0, set()
+    for code, kind in ((0, "small"), (1, "both"), (2, "large")):
+        share = float((kinds == code).mean())
+        if share == 0.0:
+            continue
+        entry = NCU_DRAM_BYTES_PER_LAUNCH.get((family, kind))
+        if entry is None:
+            return None, None
+        total += share * entry[0]
+        files.add(entry[1])
+    return total, sorted(files)
+
+
 def oracle_sample(cfg, wl, budget_s: float, max_steps: int, skip: int):
     """Times the CPU oracle as it stands on steps [skip, skip + n) of the workload, all rows.
     The oracle always starts from Algorithm 1's initial state, so the first `skip` steps
@@ -172,6 +251,40 @@ def pinned(a: np.ndarray):
     return t.pin_memory()
 
 
+def config_keys(cfg) -> dict:
+    """The `config` object: the same keys in both arms."""
+    return {"workload": cfg.name, "B": cfg.B, "V": cfg.V, "H_small": cfg.H_small, "H_large": cfg.H_large,
+            "w": cfg.w, "d_min": cfg.d_min, "tau": cfg.tau}
+
+
+class WorkloadCache:
+    """Host inputs by what determines their bits, so that configurations that differ only in
+    the threshold or the start model share one draw."""
+
+    def __init__(self):
+        self._heads, self._hidden = {}, {}
+
+    def get(self, cfg, T):
+        hk = (cfg.seed, cfg.V, cfg.H_small, cfg.H_large)
+        if hk not in self._heads:
+            self._heads = {hk: (synth.lm_head(cfg.seed, 0, cfg.V, cfg.H_small),
+                                synth.lm_head(cfg.seed, 1, cfg.V, cfg.H_large))}     # keep one pair only
+        xk = hk + (cfg.B, T, cfg.stay_easy, cfg.stay_hard, cfg.p_hard0, cfg.s_easy, cfg.s_hard)
+        if xk not in self._hidden:
+            wl = synth.Workload(cfg, T=T, heads=False)
+            self._hidden = {xk: wl}
+        h = self._hidden[xk]
+        return HostInputs(cfg, T, h.h_small, h.h_large, *self._heads[hk])
+
+
+class HostInputs:
+    """bf16 bit patterns of one configuration's inputs (host memory)."""
+
+    def __init__(self, cfg, T, h_small, h_large, W_small, W_large):
+        self.cfg, self.T = cfg, T
+        self.h_small, self.h_large, self.W_small, self.W_large = h_small, h_large, W_small, W_large
+
+
 # ----------------------------------------------------------------------------- arms
 def run_reference(args, cfg):
     rank = int(os.environ.get("RANK", "0"))
@@ -186,8 +299,7 @@ def run_reference(args, cfg):
     line = {"impl": "reference", "metric": METRIC, "value": rate, "unit": UNIT, "n_gpus": args.gpus,
             "steps": K, "warmup": W, "ms_per_step": 1e3 / rate, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "B": cfg.B, "V": cfg.V, "H_small": cfg.H_small,
-                       "H_large": cfg.H_large, "w": cfg.w, "d_min": cfg.d_min, "tau": cfg.tau},
+            "config": config_keys(cfg),
             "seq_tokens_per_s": rate * cfg.B,
             "cpu_baseline": {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": sample},
@@ -196,24 +308,45 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
-def run_ours(args, cfg):
-    import torch
-    import torch.distributed as dist
-    from paper_2502_06833_b200 import binding as E
+class Runtime:
+    """Process-wide pieces of the GPU arm: torch, the binding, the process group."""
 
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    K, W = args.steps, args.warmup
+    def __init__(self):
+        import torch
+        import torch.distributed as dist
+        from paper_2502_06833_b200 import binding as E
+        self.torch, self.dist, self.E = torch, dist, E
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+        torch.cuda.set_device(self.local)
+        if self.world > 1:
+            dist.init_process_group("nccl", device_id=torch.device("cuda", self.local))
+        self.uuid = str(torch.cuda.get_device_properties(self.local).uuid)
+        self.peaks = load_peaks()
+        self.cache = WorkloadCache()
+
+    def barrier(self):
+        if self.world > 1:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def max_over_ranks(self, ms: float, steps: int):
+        return aggregate_over_ranks(ms, steps, self.dist if self.world > 1 else None)
+
+    def close(self):
+        if self.world > 1:
+            self.dist.destroy_process_group()
+
+
+def measure(rt: Runtime, cfg, K: int, W: int, repeats: int | None, temperature: float = 0.0) -> dict:
+    """One configuration by the protocol of the module docstring.  Returns the measurements;
+    `wl` (host inputs) rides along for the CPU-oracle leg."""
+    torch, E = rt.torch, rt.E
     T_total = W + K
-    peaks = load_peaks()
-
-    wl = synth.Workload(cfg, T=T_total)
+    wl = rt.cache.get(cfg, T_total)
     hs_pin, hl_pin = pinned(wl.h_small), pinned(wl.h_large)
     W_small = pinned(wl.W_small).cuda().view(torch.bfloat16)
     W_large = pinned(wl.W_large).cuda().view(torch.bfloat16)
@@ -228,104 +361,167 @@ def run_ours(args, cfg):
     stream = torch.cuda.current_stream()
     ctx = E.ead_create(B=B, V=cfg.V, H_small=cfg.H_small, H_large=cfg.H_large, w=cfg.w,
                        d_min=cfg.d_min, tau=cfg.tau, unit=cfg.unit, start_model=cfg.start_model,
-                       W_small=W_small, W_large=W_large, device=local, stream=stream.cuda_stream)
+                       W_small=W_small, W_large=W_large, device=rt.local, stream=stream.cuda_stream,
+                       temperature=temperature, seed=cfg.seed)
 
     def outs(t0):
         return (tok[t0:], Hd[t0:], Hbar[t0:], used[t0:], nxt[t0:])
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    # ---- device-resident: W warm-up steps, then exactly K timed steps
-    E.ead_run(ctx, W, hs, hl, *outs(0))
-    barrier()
-    l0 = E.ead_kernel_launches(ctx)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    uuid = str(torch.cuda.get_device_properties(local).uuid)
-    with ClockSampler(uuid) as clocks:
+
+    # W warm-up steps; the state they leave is the start of every timed region
+    E.ead_run(ctx, W, hs, hl, *outs(0))
+    rt.barrier()
+    blob = E.ead_get_state(ctx)
+
+    def timed_device():
+        E.ead_set_state(ctx, blob)
+        rt.barrier()
         e0.record()
         E.ead_run(ctx, K, hs[W:], hl[W:], *outs(W))
         e1.record()
-        barrier()
-    launches = E.ead_kernel_launches(ctx) - l0
-    status = E.ead_status(ctx)
-    value, t_ms, world_seen = aggregate_over_ranks(e0.elapsed_time(e1), K, dist if world > 1 else None)
-    used_np = used.cpu().numpy()
+        rt.barrier()
+        return rt.max_over_ranks(e0.elapsed_time(e1), K)[1]
 
-    # ---- the LM-head kernel alone: events around every launch over the same K steps
-    E.ead_reset(ctx)
-    E.ead_run(ctx, W, hs, hl, *outs(0))
-    kms = E.ead_run_timed(ctx, K, hs[W:], hl[W:], *outs(W))
-    assert np.array_equal(used.cpu().numpy(), used_np), "timed replay diverged from the graph run"
-    bytes_s, flops_s = step_costs(cfg, used_np[W:])
-    t_kernel = kms["lmhead_ms"] * 1e-3 / K                      # seconds per launch
-    t_hbm = bytes_s.mean() / (peaks["hbm_gbs"] * 1e9)
-    t_mma = flops_s.mean() / (peaks["bf16_tflops_sustained"] * 1e12)
-    if t_hbm >= t_mma:
-        roof = {"bound": "hbm", "achieved": bytes_s.mean() / t_kernel / 1e9, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s"}
-    else:
-        roof = {"bound": "tensor", "achieved": flops_s.mean() / t_kernel / 1e12,
-                "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = NCU_TRAFFIC_BYTES_PER_LAUNCH.get(cfg.name)
-    roof.update({"kernel": "ead_lmhead_small_kernel" if B <= 128 else "ead_lmhead_kernel", "kernel_us_per_launch": t_kernel * 1e6,
-                 "algorithmic_bytes_per_launch": bytes_s.mean(), "flops_per_launch": flops_s.mean(),
-                 "peak_source": peaks["source"] + (" (sustained bf16)" if roof["bound"] == "tensor" else ""),
-                 "step_frac": (bytes_s.mean() / (t_ms * 1e-3 / K) / 1e9 / peaks["hbm_gbs"]) if roof["bound"] == "hbm"
-                 else (flops_s.mean() / (t_ms * 1e-3 / K) / 1e12 / peaks["bf16_tflops_sustained"]),
-                 "other_kernels_us_per_step": (kms["compact_ms"] + kms["merge_gate_ms"]) * 1e3 / K})
-
-    # ---- end to end through the host-buffer entry point (pinned host memory)
     o_host = [torch.empty(T_total, B, dtype=d).pin_memory()
               for d in (torch.int32, torch.float32, torch.float32, torch.uint8, torch.uint8)]
-    E.ead_reset(ctx)
-    E.ead_run_host(ctx, W, hs_pin, hl_pin, *[o[:W] for o in o_host])
-    barrier()
-    e0.record()
-    E.ead_run_host(ctx, K, hs_pin[W:], hl_pin[W:], *[o[W:] for o in o_host])
-    e1.record()
-    barrier()
-    e2e_value, _, _ = aggregate_over_ranks(e0.elapsed_time(e1), K, dist if world > 1 else None)
-    assert np.array_equal(o_host[3].numpy(), used_np), "host-buffer run diverged from the device run"
-    h2d = 2 * B * (cfg.H_small + cfg.H_large)
-    d2h = B * (4 + 4 + 4 + 1 + 1)
+
+    def timed_host():
+        E.ead_set_state(ctx, blob)
+        rt.barrier()
+        e0.record()
+        E.ead_run_host(ctx, K, hs_pin[W:], hl_pin[W:], *[o[W:] for o in o_host])
+        e1.record()
+        rt.barrier()
+        return rt.max_over_ranks(e0.elapsed_time(e1), K)[1]
+
+    with ClockSampler(rt.uuid) as clocks:
+        # ---- device-resident: exactly K timed steps per repeat
+        l0 = E.ead_kernel_launches(ctx)
+        first = timed_device()
+        launches = E.ead_kernel_launches(ctx) - l0
+        n_rep = repeats if repeats else int(min(MAX_REPEATS, max(MIN_REPEATS, math.ceil(
+            TARGET_TIMED_SECONDS * 1e3 / max(first, 1e-3)))))
+        if rt.world > 1:                                   # every rank must take the same count
+            buf = torch.tensor([n_rep], dtype=torch.int64, device="cuda")
+            rt.dist.all_reduce(buf, op=rt.dist.ReduceOp.MAX)
+            n_rep = int(buf.item())
+        dev_ms = [first] + [timed_device() for _ in range(n_rep - 1)]
+        used_np = used.cpu().numpy()
+        status = E.ead_status(ctx)
+
+        # ---- the LM-head kernel alone: events around every launch over the same K steps
+        k_rep = min(n_rep, MIN_REPEATS)
+        kern = []
+        for _ in range(k_rep):
+            E.ead_set_state(ctx, blob)
+            kern.append(E.ead_run_timed(ctx, K, hs[W:], hl[W:], *outs(W)))
+        assert np.array_equal(used.cpu().numpy(), used_np), "timed replay diverged from the graph run"
+
+        # ---- end to end through the host-buffer entry point (pinned host memory)
+        timed_host()                                       # allocates the staging buffers
+        host_ms = [timed_host() for _ in range(k_rep)]
+        assert np.array_equal(o_host[3].numpy()[W:], used_np[W:]), "host-buffer run diverged from the device run"
     info = E.ead_launch_info(ctx)
     E.ead_destroy(ctx)
 
+    t_ms = float(np.median(dev_ms))
+    bytes_s, flops_s = step_costs(cfg, used_np[W:])
+    t_kernel = float(np.median([k["lmhead_ms"] for k in kern])) * 1e-3 / K          # seconds per launch
+    roof = roofline_of(bytes_s.mean(), flops_s.mean(), t_kernel, t_ms * 1e-3 / K, rt.peaks)
+    traffic, files = ncu_traffic(cfg, used_np[W:])
+    roof["traffic"] = traffic
+    roof["traffic_source"] = files
+    roof.update({"kernel": "ead_lmhead_small_kernel" if B <= 128 else "ead_lmhead_kernel",
+                 "kernel_us_per_launch": t_kernel * 1e6,
+                 "algorithmic_bytes_per_launch": bytes_s.mean(), "flops_per_launch": flops_s.mean(),
+                 "other_kernels_us_per_step": float(np.median(
+                     [k["compact_ms"] + k["merge_gate_ms"] for k in kern])) * 1e3 / K})
+    e2e_ms = float(np.median(host_ms))
+    return {"cfg": cfg, "wl": wl, "K": K, "W": W, "temperature": temperature,
+            "world": rt.world, "ms": t_ms, "repeat_ms": dev_ms, "value": rt.world * K / (t_ms * 1e-3),
+            "e2e_value": rt.world * K / (e2e_ms * 1e-3), "e2e_repeat_ms": host_ms,
+            "h2d": 2 * B * (cfg.H_small + cfg.H_large), "d2h": B * (4 + 4 + 4 + 1 + 1),
+            "launches": int(launches), "roofline": roof, "clocks": clocks.summary(),
+            "large_head_share": float(used_np[W:].mean()), "launch": info, "status": status,
+            "weights_gb_per_step": bytes_s.mean() / 1e9}
+
+
+def per_config_entry(m: dict) -> dict:
+    cfg = m["cfg"]
+    name = cfg.name if m["temperature"] == 0.0 else f"{cfg.name}@T={m['temperature']:g}"
+    return {"workload": name, "B": cfg.B, "temperature": m["temperature"],
+            "large_head_share": m["large_head_share"], "steps": m["K"], "warmup": m["W"],
+            "repeats": len(m["repeat_ms"]), "ms_per_step": m["ms"] / m["K"],
+            "ms_per_step_min": min(m["repeat_ms"]) / m["K"], "ms_per_step_max": max(m["repeat_ms"]) / m["K"],
+            "value": m["value"], "unit": UNIT, "seq_tokens_per_s": m["value"] * cfg.B,
+            "roofline": m["roofline"],
+            "e2e": {"value": m["e2e_value"], "unit": UNIT, "h2d_bytes_per_step": m["h2d"],
+                    "d2h_bytes_per_step": m["d2h"]},
+            "clocks": m["clocks"], "gpu_launches": m["launches"], "launch": m["launch"],
+            "status_word": m["status"]}
+
+
+def run_ours(args):
+    rt = Runtime()
+    everything = args.config in (None, "all")
+    head_cfg = configs.ALL[HEADLINE if everything else args.config]
+    W = max(3, args.warmup)
+    K = args.steps if args.steps is not None else max(1, head_cfg.T - W)
+    head = measure(rt, head_cfg, K, W, args.repeats, args.temperature)
+
     # ---- CPU oracle beside it (rank 0, single GPU runs only)
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rt.rank == 0 and rt.world == 1 and not args.no_cpu_baseline:
         budget = float(args.cpu_seconds if args.cpu_seconds is not None else 15.0)
-        rate, n, dt, cores, fl = oracle_sample(cfg, wl, budget, K, skip=W)
+        rate, n, dt, cores, fl = oracle_sample(head_cfg, head["wl"], budget, K, skip=W)
         cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"steps {W}..{W + n} of the same workload, all {B} rows "
+               "sample": f"steps {W}..{W + n} of the same workload, all {head_cfg.B} rows "
                          f"(large-head share {fl:.2f}), {dt:.1f} s"}
 
-    if rank == 0:
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world_seen, "steps": K,
-                "warmup": W, "ms_per_step": t_ms / K, "higher_is_better": True, "scaling": "weak",
+    rows = []
+    if everything:
+        for name, temp in PER_CONFIG:
+            cfg = configs.ALL[name]
+            Wc = max(W, PER_CONFIG_MIN_WARMUP)
+            if args.steps is not None:
+                Kc = max(args.steps, PER_CONFIG_MIN_STEPS)
+            else:
+                Kc = 256 if cfg.B == 1 else 64
+            Kc = min(Kc, cfg.T - Wc)
+            rows.append(per_config_entry(measure(rt, cfg, Kc, Wc, args.repeats, temp)))
+
+    if rt.rank == 0:
+        roof = head["roofline"]
+        line = {"metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": head["world"], "steps": K,
+                "warmup": W, "ms_per_step": head["ms"] / K, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": cfg.name, "B": B, "V": cfg.V, "H_small": cfg.H_small,
-                           "H_large": cfg.H_large, "w": cfg.w, "d_min": cfg.d_min, "tau": cfg.tau,
-                           "large_head_share": float(used_np[W:].mean()),
-                           "l2": "inputs larger than L2: every step streams %.2f GB of weights"
-                                 % (bytes_s.mean() / 1e9),
-                           "multi_gpu": "replicas only" if world_seen > 1 else "single GPU",
-                           "launch": info},
-                "seq_tokens_per_s": value * B,
-                "clocks": clocks.summary(),
-                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                        "d2h_bytes_per_step": d2h},
-                "gpu_launches": int(launches),
+                "config": config_keys(head_cfg),
+                "temperature": args.temperature,
+                "repeats": len(head["repeat_ms"]), "repeat_ms": head["repeat_ms"],
+                "timing": "median over the repeats of one timed region of exactly `steps` steps, "
+                          "each restarted from the state after `warmup` steps; max over ranks per repeat",
+                "large_head_share": head["large_head_share"],
+                "l2": "inputs larger than L2: every step streams %.2f GB of weights" % head["weights_gb_per_step"],
+                "multi_gpu": "replicas only" if head["world"] > 1 else "single GPU",
+                "launch": head["launch"],
+                "seq_tokens_per_s": head["value"] * head_cfg.B,
+                "clocks": head["clocks"],
+                "e2e": {"value": head["e2e_value"], "unit": UNIT, "h2d_bytes_per_step": head["h2d"],
+                        "d2h_bytes_per_step": head["d2h"]},
+                "gpu_launches": head["launches"],
                 "roofline": roof,
                 "cpu_baseline": cpu,
-                "status_word": status}
+                "status_word": head["status"]}
+        if everything:
+            line["per_config"] = rows
+            line["per_config_protocol"] = (
+                "same protocol as the headline; at least %d warm-up steps so that the share of rows on the "
+                "large head is the configuration's, at least %d timed steps per repeat; fractions are of the "
+                "binding bound (copy rate, or sustained bf16 rate with the fraction of burst beside it)"
+                % (PER_CONFIG_MIN_WARMUP, PER_CONFIG_MIN_STEPS))
         print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    rt.close()
 
 
 def main():
@@ -333,20 +529,22 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=32)
-    ap.add_argument("--config", default="llama_b1", choices=sorted(configs.ALL))
+    ap.add_argument("--config", default=None, choices=sorted(configs.ALL) + ["all"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--repeats", type=int, default=None)
+    ap.add_argument("--temperature", type=float, default=0.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=None)
     args = ap.parse_args()
-    cfg = configs.ALL[args.config]
     if args.warmup < 3:
         args.warmup = 3
-    if args.steps is None:
-        args.steps = max(1, cfg.T - args.warmup)
     if args.impl == "reference":
+        cfg = configs.ALL[HEADLINE if args.config in (None, "all") else args.config]
+        if args.steps is None:
+            args.steps = max(1, cfg.T - args.warmup)
         run_reference(args, cfg)
     else:
-        run_ours(args, cfg)
+        run_ours(args)
 
 
 if __name__ == "__main__":
