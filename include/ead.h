@@ -135,13 +135,16 @@ int ead_run(ead_ctx *ctx, int32_t T, const void *h_small_seq, const void *h_larg
  * The same T steps as ead_run, but every buffer is a HOST pointer: hidden
  * states are copied to the device and results back through internal staging
  * buffers, in chunks that overlap with the computation.  Synchronous: returns
- * when the outputs are complete.  Any output may be NULL.  Pinned host memory
- * makes the copies faster but is not required.
+ * when the outputs are complete, and also when it fails: before an error is
+ * returned every copy already enqueued to or from the caller's buffers has ended.
+ * Any output may be NULL.  Pinned host memory makes the copies faster but is not required.
  */
 int ead_run_host(ead_ctx *ctx, int32_t T, const void *h_small_seq, const void *h_large_seq,
                  int32_t *tok, float *H, float *Hbar, uint8_t *model_used, uint8_t *next_model);
 
 /*
+ * DIAGNOSTIC (measurement aid, not part of the gate step's interface; so are
+ * ead_kernel_launches, ead_launch_info and ead_plan_split below).
  * The same T steps as ead_run, launched kernel by kernel (no graph replay) with
  * CUDA events around every kernel on cfg.stream, to attribute device time.
  *   kernel_ms  host, float [3]: summed device time in milliseconds of the
@@ -168,7 +171,9 @@ int ead_status(ead_ctx *ctx, uint32_t *status_word);
  * flags, number of steps taken).  ead_state_size gives the blob size for this
  * context; ead_get_state copies device -> host, ead_set_state host -> device.
  * Both wait for the stream.  A blob is only valid for a context with the same
- * B and w.  Errors: EAD_EINVALID_ARG, EAD_ESTATE, EAD_ECUDA.
+ * B and w; ead_set_state also rejects (EAD_ESTATE, nothing copied) a blob whose flags are
+ * not 0 / 1 or whose dwell counters or window fill counts are negative.
+ * Errors: EAD_EINVALID_ARG, EAD_ESTATE, EAD_ECUDA.
  */
 size_t ead_state_size(const ead_ctx *ctx);
 int ead_get_state(ead_ctx *ctx, void *host_blob, size_t size);
@@ -203,11 +208,11 @@ int ead_usage(ead_ctx *ctx, uint64_t *counts, uint32_t *per_row);
  */
 double ead_parameter_ratio(uint64_t tokens_small, uint64_t tokens_large, double P_small, double P_large);
 
-/* Number of kernels the library has launched through this context so far
+/* DIAGNOSTIC.  Number of kernels the library has launched through this context so far
  * (graph replays count their kernel nodes). */
 int64_t ead_kernel_launches(const ead_ctx *ctx);
 
-/* Launch geometry chosen at creation, for reporting: fills up to n ints with
+/* DIAGNOSTIC.  Launch geometry chosen at creation, for reporting: fills up to n ints with
  * {CTAs of the LM-head kernel, pipeline stages, rows of the hidden-state TMA
  * box, dynamic shared memory bytes}. */
 int ead_launch_info(const ead_ctx *ctx, int32_t *info, int32_t n);
@@ -283,7 +288,7 @@ int ead_shard_gate(ead_ctx *ctx, const void *all_records, int32_t n_shards, int3
                    float *Hbar, uint8_t *model_used, uint8_t *next_model);
 
 /*
- * How the LM-head kernel divides one head among its CTAs (host-side replica of the rule
+ * DIAGNOSTIC.  How the large-batch LM-head kernel divides one head among its CTAs (host-side replica of the rule
  * the kernel applies on the device; pure arithmetic, needs no GPU).  With n rows on a head
  * there are R = ceil(n / 128) row blocks; CTA `cta` of `G` serves row block out[1] and
  * vocabulary columns [out[3], out[4]) (multiples of 16; the end may exceed V by < 16).
@@ -322,7 +327,8 @@ void ead_destroy(ead_ctx *ctx);
  *   device   CUDA device ordinal; made current by the call
  *   stream   cudaStream_t to enqueue on; NULL = legacy default stream
  *
- * Asynchronous: three kernels are enqueued on `stream`.  The first call on a device also
+ * Asynchronous: four kernels are enqueued on `stream` (status clear, staging of the hidden
+ * rows, the LM-head contraction, the merge).  The first call on a device also
  * looks up the device address of the built-in array and the device's limits; make that
  * first call outside any stream capture.
  * Every call on a device uses the SAME array.  The call rewrites all of it that it later

@@ -314,12 +314,18 @@ double oracle_parameter_ratio(double usage_large, double P_small, double P_large
     return (alpha * P_small + beta * P_large) / P_large;
 }
 
-/* Tokens produced by each model and number of switches in a [T] trace of one sequence. */
-void oracle_usage(const uint8_t *used, const uint8_t *next, int64_t T, int64_t *tokens_small,
-                  int64_t *tokens_large, int64_t *switches)
+/*
+ * Tokens produced by each model and number of switches in a [T] trace of one sequence
+ * (Table 1's usage column counts generated tokens).  `tok` may be NULL; if given, a step
+ * whose token is -1 produced nothing (Algorithm 1's "while not done" had ended for the
+ * sequence, or its logits were not finite) and counts neither as a token nor as a switch.
+ */
+void oracle_usage(const uint8_t *used, const uint8_t *next, const int32_t *tok, int64_t T,
+                  int64_t *tokens_small, int64_t *tokens_large, int64_t *switches)
 {
     int64_t s = 0, l = 0, sw = 0;
     for (int64_t t = 0; t < T; ++t) {
+        if (tok && tok[t] < 0) continue;
         if (used[t]) l += 1; else s += 1;
         if (next[t] != used[t]) sw += 1;
     }

@@ -74,8 +74,9 @@ def lib():
         L.oracle_parameter_ratio.restype = C.c_double
         L.oracle_parameter_ratio.argtypes = [C.c_double, C.c_double, C.c_double]
         L.oracle_usage.restype = None
-        L.oracle_usage.argtypes = [C.POINTER(C.c_uint8), C.POINTER(C.c_uint8), C.c_int64,
-                                   C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+        L.oracle_usage.argtypes = [C.POINTER(C.c_uint8), C.POINTER(C.c_uint8), C.POINTER(C.c_int32),
+                                   C.c_int64, C.POINTER(C.c_int64), C.POINTER(C.c_int64),
+                                   C.POINTER(C.c_int64)]
         L.oracle_num_threads.restype = C.c_int
         L.oracle_num_threads.argtypes = []
         _lib = L
@@ -130,13 +131,15 @@ def parameter_ratio(usage_large: float, P_small: float, P_large: float) -> float
     return float(lib().oracle_parameter_ratio(float(usage_large), float(P_small), float(P_large)))
 
 
-def usage(used, nxt):
-    """(tokens by the small model, tokens by the large model, switches) of one [T] trace."""
+def usage(used, nxt, tok=None):
+    """(tokens by the small model, tokens by the large model, switches) of one [T] trace; with
+    ``tok`` given, steps whose token is -1 (sequence already ended) are not counted."""
     used = np.ascontiguousarray(used, dtype=np.uint8)
     nxt = np.ascontiguousarray(nxt, dtype=np.uint8)
+    tok = None if tok is None else np.ascontiguousarray(tok, dtype=np.int32)
     a, b, c = C.c_int64(), C.c_int64(), C.c_int64()
-    lib().oracle_usage(_p(used, C.c_uint8), _p(nxt, C.c_uint8), used.size, C.byref(a), C.byref(b),
-                       C.byref(c))
+    lib().oracle_usage(_p(used, C.c_uint8), _p(nxt, C.c_uint8), _p(tok, C.c_int32), used.size,
+                       C.byref(a), C.byref(b), C.byref(c))
     return int(a.value), int(b.value), int(c.value)
 
 

@@ -188,7 +188,8 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr, int shar
     cudaError_t e = cudaSuccess;
     if (ev) cudaEventRecord(ev[0], s);
     e = launch(ead_compact_kernel, dim3(cgrid), dim3(kCompactThreads), static_cast<size_t>(c.B) * sizeof(int32_t), s, pdl,
-               x->ctl, x->args, x->flag, x->done, c.B, c.H_small, c.H_large, x->hc[0], x->hc[1], x->perm);
+               x->ctl, x->args, x->flag, x->done, c.B, c.H_small, c.H_large, x->hc[0], x->hc[1], x->perm,
+               x->small_cols ? 0 : 1);
     if (e != cudaSuccess) return EAD_ECUDA;
     if (ev) cudaEventRecord(ev[1], s);
 
@@ -633,39 +634,48 @@ int ead_run_host(ead_ctx *x, int32_t T, const void *h_small_seq, const void *h_l
     const size_t row_s = static_cast<size_t>(c.B) * c.H_small * 2, row_l = static_cast<size_t>(c.B) * c.H_large * 2;
     const uint8_t *hs = static_cast<const uint8_t *>(h_small_seq), *hl = static_cast<const uint8_t *>(h_large_seq);
     const int chunks = (T + S - 1) / S;
-    for (int k = 0; k < chunks; ++k) {
+    // A failed call inside the loop must not leave copies to or from the caller's buffers in
+    // flight: every error path falls through to the synchronisation below.
+#define EAD_TRY(x)                     \
+    if (rc == EAD_OK && (x) != cudaSuccess) rc = EAD_ECUDA
+    for (int k = 0; k < chunks && rc == EAD_OK; ++k) {
         const int i = k & 1;
         const int t0 = k * S, n = std::min(S, T - t0);
         const size_t cells = static_cast<size_t>(n) * c.B;
         // inputs of chunk k -> staging buffer i, once the compute that read it (chunk k-2) is done
-        if (k >= 2) EAD_CUDA(cudaStreamWaitEvent(x->in_stream, x->ev_comp[i], 0));
-        EAD_CUDA(cudaMemcpyAsync(x->st_h[i][0], hs + t0 * row_s, n * row_s, cudaMemcpyHostToDevice, x->in_stream));
-        EAD_CUDA(cudaMemcpyAsync(x->st_h[i][1], hl + t0 * row_l, n * row_l, cudaMemcpyHostToDevice, x->in_stream));
-        EAD_CUDA(cudaEventRecord(x->ev_in[i], x->in_stream));
+        if (k >= 2) EAD_TRY(cudaStreamWaitEvent(x->in_stream, x->ev_comp[i], 0));
+        EAD_TRY(cudaMemcpyAsync(x->st_h[i][0], hs + t0 * row_s, n * row_s, cudaMemcpyHostToDevice, x->in_stream));
+        EAD_TRY(cudaMemcpyAsync(x->st_h[i][1], hl + t0 * row_l, n * row_l, cudaMemcpyHostToDevice, x->in_stream));
+        EAD_TRY(cudaEventRecord(x->ev_in[i], x->in_stream));
         // compute, once the inputs are in and the previous results of buffer i have been read back
-        EAD_CUDA(cudaStreamWaitEvent(x->stream, x->ev_in[i], 0));
-        if (k >= 2) EAD_CUDA(cudaStreamWaitEvent(x->stream, x->ev_out[i], 0));
+        EAD_TRY(cudaStreamWaitEvent(x->stream, x->ev_in[i], 0));
+        if (k >= 2) EAD_TRY(cudaStreamWaitEvent(x->stream, x->ev_out[i], 0));
         uint8_t *o = static_cast<uint8_t *>(x->st_out[i]);
-        rc = run_device(x, n, x->st_h[i][0], x->st_h[i][1], reinterpret_cast<int32_t *>(o + l.off_tok),
-                        reinterpret_cast<float *>(o + l.off_H), reinterpret_cast<float *>(o + l.off_Hbar),
-                        o + l.off_used, o + l.off_next);
-        if (rc != EAD_OK) return rc;
-        EAD_CUDA(cudaEventRecord(x->ev_comp[i], x->stream));
+        if (rc == EAD_OK)
+            rc = run_device(x, n, x->st_h[i][0], x->st_h[i][1], reinterpret_cast<int32_t *>(o + l.off_tok),
+                            reinterpret_cast<float *>(o + l.off_H), reinterpret_cast<float *>(o + l.off_Hbar),
+                            o + l.off_used, o + l.off_next);
+        EAD_TRY(cudaEventRecord(x->ev_comp[i], x->stream));
         // results of chunk k -> host
-        EAD_CUDA(cudaStreamWaitEvent(x->out_stream, x->ev_comp[i], 0));
+        EAD_TRY(cudaStreamWaitEvent(x->out_stream, x->ev_comp[i], 0));
         const size_t o0 = static_cast<size_t>(t0) * c.B;
-        if (tok) EAD_CUDA(cudaMemcpyAsync(tok + o0, o + l.off_tok, 4 * cells, cudaMemcpyDeviceToHost, x->out_stream));
-        if (H) EAD_CUDA(cudaMemcpyAsync(H + o0, o + l.off_H, 4 * cells, cudaMemcpyDeviceToHost, x->out_stream));
-        if (Hbar) EAD_CUDA(cudaMemcpyAsync(Hbar + o0, o + l.off_Hbar, 4 * cells, cudaMemcpyDeviceToHost, x->out_stream));
+        if (tok) EAD_TRY(cudaMemcpyAsync(tok + o0, o + l.off_tok, 4 * cells, cudaMemcpyDeviceToHost, x->out_stream));
+        if (H) EAD_TRY(cudaMemcpyAsync(H + o0, o + l.off_H, 4 * cells, cudaMemcpyDeviceToHost, x->out_stream));
+        if (Hbar) EAD_TRY(cudaMemcpyAsync(Hbar + o0, o + l.off_Hbar, 4 * cells, cudaMemcpyDeviceToHost, x->out_stream));
         if (model_used)
-            EAD_CUDA(cudaMemcpyAsync(model_used + o0, o + l.off_used, cells, cudaMemcpyDeviceToHost, x->out_stream));
+            EAD_TRY(cudaMemcpyAsync(model_used + o0, o + l.off_used, cells, cudaMemcpyDeviceToHost, x->out_stream));
         if (next_model)
-            EAD_CUDA(cudaMemcpyAsync(next_model + o0, o + l.off_next, cells, cudaMemcpyDeviceToHost, x->out_stream));
-        EAD_CUDA(cudaEventRecord(x->ev_out[i], x->out_stream));
+            EAD_TRY(cudaMemcpyAsync(next_model + o0, o + l.off_next, cells, cudaMemcpyDeviceToHost, x->out_stream));
+        EAD_TRY(cudaEventRecord(x->ev_out[i], x->out_stream));
     }
-    EAD_CUDA(cudaStreamSynchronize(x->out_stream));
-    EAD_CUDA(cudaStreamSynchronize(x->stream));
-    return EAD_OK;
+#undef EAD_TRY
+    // the call is synchronous, also when it fails
+    const cudaError_t s_in = cudaStreamSynchronize(x->in_stream);
+    const cudaError_t s_comp = cudaStreamSynchronize(x->stream);
+    const cudaError_t s_out = cudaStreamSynchronize(x->out_stream);
+    if (rc == EAD_OK && (s_in != cudaSuccess || s_comp != cudaSuccess || s_out != cudaSuccess)) rc = EAD_ECUDA;
+    if (rc != EAD_OK) cudaGetLastError();
+    return rc;
 }
 
 int ead_shard_range(int32_t V, int32_t n_shards, int32_t shard, int32_t *begin, int32_t *end)
@@ -794,6 +804,15 @@ int ead_set_state(ead_ctx *x, const void *blob, size_t size)
     p += sizeof hd;
     for (size_t i = 0; i < B; ++i)
         if (p[i] > 1 || p[B + pad + i] > 1) return EAD_ESTATE;
+    {
+        // dwell counters and window fill counts index device arrays: a negative one is not a state
+        const uint8_t *q = p + 2 * (B + pad);
+        for (size_t i = 0; i < 2 * B; ++i) {
+            int32_t v;
+            memcpy(&v, q + 4 * i, 4);
+            if (v < 0) return EAD_ESTATE;
+        }
+    }
     EAD_CUDA(cudaMemcpy(&x->ctl->step, &hd.step, 4, cudaMemcpyHostToDevice));
     EAD_CUDA(cudaMemcpy(x->flag, p, B, cudaMemcpyHostToDevice));
     p += B + pad;

@@ -49,7 +49,7 @@ __global__ void ead_reset_kernel(StepCtl *ctl, uint8_t *flag, int32_t *c, int32_
 // blockIdx.x + gridDim.x, ...   perm[m * B + r] = original row of compacted row r of head m.
 __global__ void __launch_bounds__(kCompactThreads)
 ead_compact_kernel(StepCtl *ctl, const RunArgs *args, const uint8_t *flag, const uint8_t *done, int B, int Hs,
-                   int Hl, uint16_t *hc_s, uint16_t *hc_l, int32_t *perm)
+                   int Hl, uint16_t *hc_s, uint16_t *hc_l, int32_t *perm, int zero_pad)
 {
     extern __shared__ uint32_t pos_sh[];         // [B]: position | class << 30 (0 small, 1 large, 2 done)
     __shared__ int32_t warp_tot[kCompactThreads / 32];
@@ -120,6 +120,25 @@ ead_compact_kernel(StepCtl *ctl, const RunArgs *args, const uint8_t *flag, const
         const uint4 *src = reinterpret_cast<const uint4 *>(args->h[f] + (static_cast<size_t>(idx) * B + b) * H);
         uint4 *dst = reinterpret_cast<uint4 *>((f ? hc_l : hc_s) + static_cast<size_t>(pos) * H);
         for (int k = tid; k < H / 8; k += kCompactThreads) dst[k] = __ldg(src + k);
+    }
+
+    // Large-batch LM-head kernel: a head's last row block is multiplied as a whole 128-row tile.
+    // The rows between the head's last real row and the end of that block would otherwise hold
+    // hidden states of earlier steps; they never reach an output either way, but the tensor
+    // cores draw power by the bits that toggle, and under the power cap a block padded with
+    // zeros runs at a higher clock than one padded with old data.
+    if (zero_pad) {
+        const int total_large = total & 0xffff, total_done = total >> 16;
+        const int n_m[2] = {B - total_large - total_done, total_large};
+        const int pad_s = (kTileM - n_m[0] % kTileM) % kTileM;
+        const int pad_l = (kTileM - n_m[1] % kTileM) % kTileM;
+        for (int q = blockIdx.x; q < pad_s + pad_l; q += gridDim.x) {
+            const int f = q < pad_s ? 0 : 1;
+            const int row = n_m[f] + (f ? q - pad_s : q);
+            const int H = f ? Hl : Hs;
+            uint4 *dst = reinterpret_cast<uint4 *>((f ? hc_l : hc_s) + static_cast<size_t>(row) * H);
+            for (int k = tid; k < H / 8; k += kCompactThreads) dst[k] = make_uint4(0u, 0u, 0u, 0u);
+        }
     }
 }
 
@@ -243,11 +262,12 @@ __device__ __forceinline__ void finish_row(const GateParams &p, const RowState &
     st.ring_global[slot] = H;
     nf += 1;
     const int cnt = nf < p.w ? nf : p.w;
+    if (nf >= 2 * p.w) nf -= p.w;                  // same slot sequence, and the counter stays bounded
     float sum = 0.f;
     for (int k = 0; k < cnt; ++k) sum += (k == slot) ? H : st.ring[k];     // slot order, as stored
     const float Hbar = sum / static_cast<float>(cnt);
     // ---- c <- c + 1; Eq. 4
-    int c = st.c + 1;
+    int c = st.c < (1 << 30) ? st.c + 1 : st.c;   // saturates far above any d_min instead of wrapping
     const int used = model;
     if (c >= p.d_min) {
         if (model == 0 && Hbar > p.tau) { model = 1; c = 0; }

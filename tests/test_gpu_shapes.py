@@ -41,6 +41,10 @@ SHAPES = [
     (8, 40000, 128, 64),          # several 256-wide tiles per CTA; large head narrower than small
     (130, 3000, 64, 128),         # two row blocks, the second with 2 rows
     (300, 5000, 128, 256),        # three row blocks shared by both heads
+    (150, 2000, 64, 128),         # one pair block per head, the second CTA of each pair mostly without rows
+    (256, 2500, 128, 64),         # both heads together fill exactly one pair block
+    (520, 1500, 64, 64),          # up to three pair blocks on one head, ragged last vocabulary tile
+    (700, 9000, 192, 320),        # full 256-wide tiles for every pair, hidden sizes that are multiples of 64
     (128, 2048, 64, 64),          # exactly one full row block
     (100, 2300, 128, 64),         # four chunks of sequences in the 17..128 variant, the last ragged
     (17, 700, 64, 128),           # smallest batch of that variant
@@ -118,6 +122,17 @@ def test_checkpoint_and_resume():
         with pytest.raises(g.E.EadError) as err:
             g.E.ead_set_state(g.ctx, blob[:-4])
         assert err.value.code == g.E.EAD_ESTATE
+        # a damaged blob: a negative window fill count or dwell counter would index outside the
+        # row's window on the device; it must be refused and leave the context as it was
+        pad = (4 - cfg.B % 4) % 4
+        off_c = 16 + 2 * (cfg.B + pad)
+        for off in (off_c + 4 * 2, off_c + 4 * cfg.B + 4 * 3):          # c[2], nfill[3]
+            bad = bytearray(blob)
+            bad[off:off + 4] = np.int32(-1).tobytes()
+            with pytest.raises(g.E.EadError) as err:
+                g.E.ead_set_state(g.ctx, bytes(bad))
+            assert err.value.code == g.E.EAD_ESTATE
+        assert g.E.ead_get_state(g.ctx)[16:] != blob[16:]                # the rest of the run moved it on
     for k in ("tok", "H", "Hbar", "used", "next"):
         assert np.array_equal(full[k][17:], rest[k]), k
 
@@ -287,6 +302,12 @@ def test_end_of_sequence_token_and_done_mask(B, V):
     with GpuGate(cfg, wl.W_small, wl.W_large, eos_token=eos) as g:
         out = g.run(wl.h_small, wl.h_large, "run")
         assert np.array_equal(g.E.ead_get_done(g.ctx, B).astype(bool), ended)
+        # usage counts generated tokens only: the steps after a row's end are in neither count
+        per_row = np.zeros((3, B), dtype=np.uint32)
+        tot = g.E.ead_usage(g.ctx, per_row)
+        want = [O.usage(ora["used"][:, b], ora["next"][:, b], ora["tok"][:, b]) for b in range(B)]
+        assert per_row.T.tolist() == [list(w) for w in want]
+        assert tot["tokens_small"] + tot["tokens_large"] == int((ora["tok"] >= 0).sum()) < B * cfg.T
         blob = g.E.ead_get_state(g.ctx)
         # a row marked done by the caller stops as well; reset clears the mask
         g.E.ead_reset(g.ctx)

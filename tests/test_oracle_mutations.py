@@ -67,6 +67,8 @@ MUTANTS = [
     ("end_of_sequence_stops_the_row_one_token_early",
      "if (eos_token >= 0 && tk == eos_token) done = 1;",
      "if (eos_token >= 0 && tk == eos_token) { done = 1; if (tok) tok[o] = -1; }"),
+    ("usage_counts_steps_after_the_sequence_ended",
+     "if (tok && tok[t] < 0) continue;", "if (tok && tok[t] < -1) continue;"),
     ("switch_count_counts_the_steps_without_a_switch",
      "if (next[t] != used[t]) sw += 1;", "if (next[t] == used[t]) sw += 1;"),
 ]

@@ -352,6 +352,19 @@ def test_usage_counts_of_hand_traces():
     assert O.usage(out["used"], out["next"]) == (5, 7, 3)
 
 
+def test_usage_counts_only_generated_tokens():
+    """Table 1's usage column is a share of generated tokens, and Algorithm 1 generates none once
+    "while not done" has ended.  Hand trace: six steps, used SSLLLL, next SLLLLL, the fourth token
+    is the last one (steps five and six report token -1): 2 small tokens, 2 large ones and the
+    one switch; without the token trace all six steps count."""
+    used, nxt = [0, 0, 1, 1, 1, 1], [0, 1, 1, 1, 1, 1]
+    assert O.usage(used, nxt, [5, 7, 2, 9, -1, -1]) == (2, 2, 1)
+    assert O.usage(used, nxt) == (2, 4, 1)
+    # an ended row reports its frozen model as used = next, so only token counts can differ;
+    # a step that produced nothing is no switch either (constructed: next differs on a dead step)
+    assert O.usage([0, 0, 0], [0, 0, 1], [3, -1, -1]) == (1, 0, 0)
+
+
 # ---------------------------------------------------------------- sampling (Algorithm 1, sampling lines)
 def test_philox_known_answers():
     """Known-answer vectors of Philox4x32-10 published with the Random123 library."""

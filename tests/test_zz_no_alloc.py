@@ -6,17 +6,37 @@ or in a latency-critical section where cudaMalloc's implicit synchronisation is 
 acceptable.  `ead_head_entropy_static` serves them from a scratch array compiled into the
 library.  This test calls it through the C ABI twice in a row (the second call with fewer
 rows and other data, so that anything left in the shared scratch by the first call would
-show) and checks tokens and entropies against `ead_step` on the same inputs, with the
-tolerance of the other parity tests.  It is collected last on purpose.
+show) and checks tokens and entropies against `ead_step` on the same inputs and against the
+CPU oracle, with the tolerance of the other parity tests; further cases run it at the limits
+its scratch array is sized for.  It is collected last on purpose.
 """
 import numpy as np
 import pytest
 
+from oracle import ead_oracle as O
 from workloads import synth
 
 pytestmark = pytest.mark.gpu
 
 H_TOL_NATS = 2e-3
+GAP_TIE = 1e-3
+
+
+def _oracle_rows(Wb, hb):
+    """Entropy (nats), greedy token and top-2 logit gap of every row by the CPU oracle."""
+    out = []
+    for row in hb:
+        z = O.logits(Wb, row)
+        tok, gap = O.greedy(z)
+        out.append((O.entropy(z), tok, gap))
+    return out
+
+
+def _check_against_oracle(tok, Hh, want):
+    tok, Hh = tok.cpu().numpy(), Hh.cpu().numpy()
+    for b, (H_o, tok_o, gap) in enumerate(want):
+        assert abs(float(Hh[b]) - H_o) <= H_TOL_NATS, (b, Hh[b], H_o)
+        assert tok[b] == tok_o or gap < GAP_TIE, (b, tok[b], tok_o, gap)
 
 
 def _bf16(bits):
@@ -63,12 +83,51 @@ def test_static_entry_point_matches_ead_step_twice():
     torch.cuda.synchronize()
     assert torch.cuda.mem_get_info()[0] == free_before      # nothing was allocated by the call
 
-    for (tok, Hh, st), (wtok, wH), B in zip(outs, want, (B1, B2)):
+    for (tok, Hh, st), (wtok, wH), B, hb in zip(outs, want, (B1, B2), (h1, h2)):
         assert st.item() == 0
         assert tok.cpu().numpy().tolist() == wtok[:B].tolist()
         np.testing.assert_allclose(Hh.cpu().numpy(), wH[:B], rtol=0, atol=H_TOL_NATS)
+        _check_against_oracle(tok, Hh, _oracle_rows(Wb, hb[:B]))
     # the two calls saw different data: easy rows first, hard rows second
     assert want[0][1].max() < want[1][1].min()
+
+
+@pytest.mark.parametrize("B,V,H", [
+    (128, 3000, 256),      # the largest batch: every row of the padded operand is a real one
+    (4, 2100, 8192),       # the longest hidden row: the staged rows fill the scratch array's width
+    (128, 700, 8192),      # both at once: the scratch layout at its tightest
+    (20, 40000, 200),      # full 256-column weight tiles and a hidden size that is no multiple of 64
+])
+def test_static_entry_point_at_its_limits_matches_the_oracle(B, V, H):
+    """Two calls in a row at the sizes the built-in scratch is dimensioned for, the second on
+    other data and fewer rows; both against the CPU oracle."""
+    import torch
+    from paper_2502_06833_b200 import binding as E
+
+    Wb = synth.lm_head(77, 0, V, H)
+    rng = np.random.default_rng(B * 1000003 + H)
+    hA = synth.f32_to_bf16_bits((3.0 * rng.normal(0, 1, (B, H))).astype(np.float32))
+    B2 = max(1, B - 3)
+    hB = synth.f32_to_bf16_bits((1.0 * rng.normal(0, 1, (B2, H))).astype(np.float32))
+    W = _bf16(Wb)
+    stream = torch.cuda.current_stream().cuda_stream
+    dev = torch.cuda.current_device()
+    results = []
+    for hb in (hA, hB):
+        n = hb.shape[0]
+        tok = torch.full((n,), -7, dtype=torch.int32, device="cuda")
+        Hh = torch.full((n,), -7.0, dtype=torch.float32, device="cuda")
+        st = torch.full((1,), 99, dtype=torch.int32, device="cuda")
+        d = _bf16(hb)
+        E.ead_head_entropy_static(W, d, n, V, H, tok, Hh, st, dev, stream)
+        results.append((tok, Hh, st, hb, d))
+    torch.cuda.synchronize()
+    rows = np.unique(np.linspace(0, B2 - 1, 12).astype(int))           # a sample keeps the oracle quick
+    for tok, Hh, st, hb, _ in results:
+        assert st.item() == 0
+        want = _oracle_rows(Wb, hb[rows])
+        _check_against_oracle(tok[rows], Hh[rows], want)
+        assert (Hh.cpu().numpy() >= 0).all() and (tok.cpu().numpy() >= 0).all() and tok.max().item() < V
 
 
 def test_static_entry_point_rejects_sizes_beyond_its_scratch():
