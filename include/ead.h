@@ -246,8 +246,9 @@ int ead_launch_info(const ead_ctx *ctx, int32_t *info, int32_t n);
  * From then on ead_step / ead_run / ead_run_host work as on one GPU, called on every shard with
  * the same hidden states: after its cross-CTA merge each shard stores its B records straight
  * into all n exchange buffers (plain stores; the record's step word last, with release
- * semantics at system scope), and a fourth kernel waits until the records of all n shards for
- * this step have arrived in the local buffer and finishes the step.  Buffers alternate with
+ * semantics at system scope), and the thread that stored a row's record then waits until that
+ * row's records of all n shards for this step have arrived in the local buffer and finishes
+ * the row: a sharded step is the same three kernels as an unsharded one.  Buffers alternate with
  * the parity of the step, which suffices because a shard cannot run more than one step ahead
  * of another.  The wait is bounded (2 s): a shard that never delivers sets
  * EAD_STATUS_WAIT_EXPIRED, the rows are reported like non-finite rows, and later steps do not

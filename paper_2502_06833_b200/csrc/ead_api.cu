@@ -178,8 +178,8 @@ GateParams gate_params(const ead_ctx *x, int reduce_only)
 // boundaries between the kernels are recorded for timing and the kernels do not overlap;
 // otherwise each kernel's set-up overlaps the tail of the one before it.
 // shard_mode (vocabulary-sharded contexts): 1 = stop after the merge, records to the caller's
-// buffer; 2 = records into every shard's exchange buffer, then a fourth kernel that waits for
-// all shards' records and finishes the step; 3 = as 2 without the fourth kernel.
+// buffer; 2 = records into every shard's exchange buffer, then the same thread waits for the
+// row's records of all shards and finishes the step; 3 = as 2 without the second half.
 int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr, int shard_mode = 0)
 {
     const ead_config &c = x->cfg;
@@ -243,7 +243,7 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr, int shar
     if (e != cudaSuccess) return EAD_ECUDA;
     if (ev) cudaEventRecord(ev[2], s);
 
-    const GateParams gp = gate_params(x, shard_mode == 3 ? 2 : shard_mode);
+    const GateParams gp = gate_params(x, shard_mode == 3 ? 2 : shard_mode == 2 ? 3 : shard_mode);
     const int rows_per_block = kGateThreads / 32;
     if (x->small_cols)
         e = launch(ead_merge_gate_wide_kernel, dim3(c.B), dim3(kGateThreads), 0, s, pdl, gp);
@@ -252,16 +252,11 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr, int shar
                    pdl, gp);
     if (e != cudaSuccess) return EAD_ECUDA;
     if (ev) cudaEventRecord(ev[3], s);
-    if (shard_mode == 2) {
-        e = launch(ead_shard_gate_kernel, dim3((c.B + 127) / 128), dim3(128), 0, s, pdl, gate_params(x, 0),
-                   static_cast<const ShardRecord *>(nullptr), 0, RunArgs{}, 2);
-        if (e != cudaSuccess) return EAD_ECUDA;
-    }
     return cudaGetLastError() == cudaSuccess ? EAD_OK : EAD_ECUDA;
 }
 
 int step_mode(const ead_ctx *x) { return x->cfg.shard_count > 0 ? 2 : 0; }
-int kernels_per_step(const ead_ctx *x) { return x->cfg.shard_count > 0 ? 4 : 3; }
+int kernels_per_step(const ead_ctx *) { return 3; }
 // Sharded contexts take whole steps only once their exchange buffers are known.
 bool can_step(const ead_ctx *x) { return x->cfg.shard_count == 0 || x->connected; }
 

@@ -161,10 +161,11 @@ struct GateParams {
     uint32_t *usage;           // [3][B]: tokens by the small model, by the large model, switches
     uint8_t *done;             // [B]: the sequence has produced the end-of-sequence token
     int32_t eos_token;         // < 0: none
-    // vocabulary-sharded use: the merge kernels stop after the cross-CTA merge and hand on one
-    // ShardRecord per row (indices shifted by v_off of the row's head): reduce_only = 1 writes
-    // it to args->shard_out (the caller exchanges), 2 stores it into the exchange buffer of
-    // every shard named in `link` (peer memory)
+    // vocabulary-sharded use: after the cross-CTA merge the kernels hand on one ShardRecord per
+    // row (indices shifted by v_off of the row's head): reduce_only = 1 writes it to
+    // args->shard_out and stops (the caller exchanges), 2 stores it into the exchange buffer of
+    // every shard named in `link` (peer memory) and stops, 3 stores it likewise, then waits for
+    // the row's records of all shards and finishes the step
     int32_t reduce_only;
     int32_t v_off[2];
     const ShardLink *link;
@@ -179,6 +180,38 @@ __device__ __forceinline__ uint32_t ld_acquire_sys(const int32_t *p)
 __device__ __forceinline__ void st_release_sys(int32_t *p, int32_t v)
 {
     asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// Vocabulary-sharded use: folds the records that the n shards delivered for sequence b and
+// exchange step `step1` (shard order) into acc / draw.  With `patient` the thread first waits
+// for each record's step word (bounded: one deadline for all its waits; an expiry sets
+// EAD_STATUS_WAIT_EXPIRED and ends the patience).  Returns whether every record belongs to
+// this step and to the head `model`.
+__device__ __forceinline__ bool gather_shard_records(const GateParams &p, const ShardRecord *all, int n_shards, int b,
+                                                     int model, int step1, bool patient, Partial &acc, Draw &draw)
+{
+    bool agree = true;
+    const unsigned long long t0 = patient ? globaltimer_ns() : 0ull;
+    for (int s = 0; s < n_shards; ++s) {
+        const ShardRecord *rec = all + static_cast<size_t>(s) * p.B + b;
+        int got = static_cast<int>(ld_acquire_sys(&rec->step1));
+        while (got != step1 && patient) {
+            __nanosleep(64);
+            got = static_cast<int>(ld_acquire_sys(&rec->step1));
+            if (got != step1 && globaltimer_ns() - t0 > kWaitLimitNs) {
+                atomicOr(&p.ctl->status, kStatusWaitExpired);
+                patient = false;
+            }
+        }
+        // ordinary loads: the acquire above orders them after the writer's release of the step word
+        const float4 lo = *reinterpret_cast<const float4 *>(rec);
+        const float2 hi = *reinterpret_cast<const float2 *>(&rec->k);
+        const int rmodel = rec->model;
+        agree = agree && got == step1 && rmodel == model;
+        acc = merge_partial(acc, Partial{lo.x, lo.y, lo.z, __float_as_int(lo.w)});
+        draw = merge_draw(draw, Draw{hi.x, __float_as_int(hi.y)});
+    }
+    return agree;
 }
 
 // Everything after the merge for one compacted row (executed by one thread): Eq. 2 in the
@@ -205,9 +238,11 @@ __device__ __forceinline__ RowState load_row_state(const GateParams &p, int m, i
     return st;
 }
 
-__device__ __forceinline__ void finish_row(const GateParams &p, const RowState &st, const Partial &acc, int t_step,
-                                           const Draw &draw, const RunArgs &out)
+__device__ __forceinline__ void finish_row(const GateParams &p, const RowState &st, const Partial &acc_in, int t_step,
+                                           const Draw &draw_in, const RunArgs &out)
 {
+    Partial acc = acc_in;
+    Draw draw = draw_in;
     if (p.reduce_only) {                          // one vocabulary shard: hand the slice's statistics on
         const int off = p.v_off[st.model];
         const int step1 = p.ctl->cur_x + 1;
@@ -235,7 +270,18 @@ __device__ __forceinline__ void finish_row(const GateParams &p, const RowState &
             dst->model = st.model;
         }
         for (int d = 0; d < lk.n; ++d) st_release_sys(&(lk.all[d] + slot)->step1, step1);
-        return;
+        if (p.reduce_only == 2) return;           // the caller runs the step's second half apart
+        // Whole step in this kernel: wait for the row's records of all shards in the local
+        // buffer, fold them in shard order (every shard folds the same values in the same
+        // order) and carry on as on one GPU.
+        acc = Partial{kNegSentinel, 0.f, 0.f, 0x7fffffff};
+        draw = Draw{-INFINITY, 0x7fffffff};
+        const ShardRecord *all = lk.all[lk.self] + static_cast<size_t>((step1 - 1) & 1) * lk.n * p.B;
+        const bool patient = !(p.ctl->status & kStatusWaitExpired);   // none at all once a wait has expired
+        if (!gather_shard_records(p, all, lk.n, st.b, st.model, step1, patient, acc, draw)) {
+            atomicOr(&p.ctl->status, kStatusShardMismatch);          // a shard is on another step or saw other flags
+            acc.s = 0.f;                                              // reported like a non-finite row: state untouched
+        }
     }
     // ---- Eq. 2 in the fused form  H = ln Z - E_p[z] = ln s - t / (s log2 e)   (nats)
     float H = logf(acc.s) - acc.t / (acc.s * kLog2e);
@@ -325,7 +371,8 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const Gate
     const int nd = p.ctl->n_done;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         if (n0 + n1 + nd != p.B) atomicOr(&p.ctl->status, kStatusBadCount);
-        if (!p.reduce_only) p.ctl->step = t_step + 1;   // nobody in this kernel reads `step`
+        if (!p.reduce_only || p.reduce_only == 3) p.ctl->step = t_step + 1;   // nobody in this kernel reads `step`
+        if (p.reduce_only == 3) p.ctl->xstep = p.ctl->cur_x + 1;
     }
     if (i >= n0 + n1 || n0 + n1 + nd != p.B) return;
     const int m = i < n0 ? 0 : 1;
@@ -381,7 +428,8 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_wide_kernel(const
     griddep_wait();                              // partials of the LM-head kernel
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         if (n0 + n1 + nd != p.B) atomicOr(&p.ctl->status, kStatusBadCount);
-        if (!p.reduce_only) p.ctl->step = t_step + 1;
+        if (!p.reduce_only || p.reduce_only == 3) p.ctl->step = t_step + 1;
+        if (p.reduce_only == 3) p.ctl->xstep = p.ctl->cur_x + 1;
     }
     if (!live) return;
     const size_t base = (static_cast<size_t>(m) * p.B + r) * p.slots_stride;
@@ -454,29 +502,9 @@ ead_shard_gate_kernel(const GateParams p, const ShardRecord *all, int n_shards, 
     }
     Partial acc{kNegSentinel, 0.f, 0.f, 0x7fffffff};
     Draw draw{-INFINITY, 0x7fffffff};
-    bool agree = true;
     // one deadline for all of this thread's waits; none at all once a wait has expired before
-    bool patient = mode >= 2 && !(p.ctl->status & kStatusWaitExpired);
-    const unsigned long long t0 = patient ? globaltimer_ns() : 0ull;
-    for (int s = 0; s < n_shards; ++s) {
-        const ShardRecord *rec = all + static_cast<size_t>(s) * p.B + b;
-        int got = static_cast<int>(ld_acquire_sys(&rec->step1));
-        while (got != step1 && patient) {
-            __nanosleep(64);
-            got = static_cast<int>(ld_acquire_sys(&rec->step1));
-            if (got != step1 && globaltimer_ns() - t0 > kWaitLimitNs) {
-                atomicOr(&p.ctl->status, kStatusWaitExpired);
-                patient = false;
-            }
-        }
-        // ordinary loads: the acquire above orders them after the writer's release of the step word
-        const float4 lo = *reinterpret_cast<const float4 *>(rec);
-        const float2 hi = *reinterpret_cast<const float2 *>(&rec->k);
-        const int rmodel = rec->model;
-        agree = agree && got == step1 && rmodel == model;
-        acc = merge_partial(acc, Partial{lo.x, lo.y, lo.z, __float_as_int(lo.w)});
-        draw = merge_draw(draw, Draw{hi.x, __float_as_int(hi.y)});
-    }
+    const bool patient = mode >= 2 && !(p.ctl->status & kStatusWaitExpired);
+    const bool agree = gather_shard_records(p, all, n_shards, b, model, step1, patient, acc, draw);
     if (!agree) {                                 // a shard is on another step or saw other flags
         atomicOr(&p.ctl->status, kStatusShardMismatch);
         acc.s = 0.f;                              // reported like a non-finite row: state untouched

@@ -80,16 +80,20 @@ class VocabParallelGate:
         self.exchange = exchange                                 # keep the mappings alive
         self.connected = True
 
-    def connect_symmetric(self) -> None:
+    def connect_symmetric(self, symm=None) -> None:
         """Allocates the exchange buffers in ``torch`` symmetric memory (peer-mapped over NVLink)
-        and connects to them.  Collective over the group."""
-        import torch.distributed._symmetric_memory as symm
+        and connects to them.  Collective over the group.  ``symm``: the symmetric-memory module
+        (default ``torch.distributed._symmetric_memory``)."""
+        if symm is None:
+            import torch.distributed._symmetric_memory as symm
         torch, dist = self.torch, self.dist
         nbytes = self.E.ead_shard_exchange_bytes(self.B, self.world)
-        buf = symm.empty(nbytes, dtype=torch.uint8, device=self.records.device)
+        dev = self.records.device
+        buf = symm.empty(nbytes, dtype=torch.uint8, device=dev)
         handle = symm.rendezvous(buf, dist.group.WORLD if self.group is None else self.group)
         buf.zero_()
-        torch.cuda.synchronize(self.records.device)
+        if getattr(dev, "type", "cpu") == "cuda":
+            torch.cuda.synchronize(dev)
         dist.barrier(group=self.group)                           # nobody stores before everybody has cleared
         self._symm = (buf, handle)
         self.connect([int(handle.buffer_ptrs[r]) for r in range(self.world)])

@@ -258,3 +258,194 @@ def test_vocab_parallel_glue_over_two_gloo_ranks(tmp_path):
     res = subprocess.run(cmd, capture_output=True, text=True, timeout=240)
     assert res.returncode == 0, res.stdout + res.stderr
     assert res.stdout.count("ok") == 2
+
+
+# The same two ranks through the other route: exchange buffers that every rank can address
+# (here: files mapped by both processes), `connect()` with one buffer per rank in rank order,
+# then whole steps by `run()`.  The stand-in engine stores its record into every rank's buffer,
+# step word last, and polls its own buffer for the others', as the CUDA kernels do.
+_VP_CONNECTED_WORKER = r"""
+import os, sys, time
+sys.path.insert(0, {root!r})
+import numpy as np, torch, torch.distributed as dist
+from paper_2502_06833_b200 import binding, vocab_parallel as VP
+from oracle import ead_oracle as O
+
+LOG2E = 1.4426950408889634
+TMP = {tmp!r}
+
+class FakeEngine:
+    EAD_SHARD_RECORD_BYTES = 32
+    ead_shard_range = staticmethod(binding.ead_shard_range)
+    def ead_shard_exchange_bytes(self, B, n):
+        return 2 * n * B * 32
+    def ead_create(self, **kw):
+        self.kw, self.xstep, self.connected_to = kw, 0, None
+        return self
+    def ead_shard_connect(self, ctx, shard, exchange):
+        assert len(exchange) == self.kw["shard_count"]
+        self.shard, self.connected_to, self.xstep = shard, list(exchange), 0
+    def _record(self, h_small):
+        W, off = self.kw["W_small"].double().numpy(), self.kw["vocab_offset_small"]
+        z = h_small.double().numpy() @ W.T
+        m = z.max(1)
+        e = np.exp(z - m[:, None])
+        rec = np.zeros((z.shape[0], 8), dtype=np.float32)
+        rec[:, 0], rec[:, 1], rec[:, 2] = m, e.sum(1), (e * (z - m[:, None])).sum(1) * LOG2E
+        rec.view(np.int32)[:, 3] = z.argmax(1) + off
+        return rec
+    def ead_step(self, ctx, h_small, h_large, tok, H, Hbar, used, nxt):
+        n, B = self.kw["shard_count"], self.kw["B"]
+        rec, step1, par = self._record(h_small), self.xstep + 1, self.xstep & 1
+        for buf in self.connected_to:                       # every shard's buffer, own one included
+            v = buf.reshape(2, n, B, 8)
+            v[par, self.shard, :, :7] = rec[:, :7]
+            buf.flush()
+            v.view(np.int32)[par, self.shard, :, 7] = step1  # the step word goes last
+            buf.flush()
+        mine = self.connected_to[self.shard].reshape(2, n, B, 8)
+        t0 = time.time()
+        while not (mine.view(np.int32)[par, :, :, 7] == step1).all():
+            assert time.time() - t0 < 60, "a shard never delivered"
+            time.sleep(0.001)
+        a, ai = mine[par].astype(np.float64), mine.view(np.int32)[par]
+        for b in range(B):
+            m, s, t, idx = -1e30, 0.0, 0.0, 2**31 - 1
+            for r in range(n):
+                qm, qs, qt, qi = a[r, b, 0], a[r, b, 1], a[r, b, 2], int(ai[r, b, 3])
+                M = max(m, qm)
+                da, db = (m - M) * LOG2E, (qm - M) * LOG2E
+                ea, eb = 2.0 ** da, 2.0 ** db
+                s, t = ea * s + eb * qs, ea * (da * s + t) + eb * (db * qs + qt)
+                idx = idx if m > qm else qi if qm > m else min(idx, qi)
+                m = M
+            H[b] = np.log(s) - t / (s * LOG2E)
+            tok[b] = idx
+        self.xstep += 1
+    def ead_run(self, ctx, T, hs, hl, tok, H, Hbar, used, nxt):
+        for t in range(T):
+            self.ead_step(ctx, hs[t], hl[t], tok[t], H[t], None, None, None)
+    def ead_destroy(self, ctx): pass
+
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+rng = np.random.default_rng(7)
+V, Hd, B, T = 1100, 32, 3, 5
+W = torch.from_numpy(rng.integers(-24, 25, (V, Hd)) / 16.0).float()
+h = torch.from_numpy(rng.integers(-16, 17, (T, B, Hd)) / 8.0).float()
+Wl = torch.zeros((V, 8))
+eng = FakeEngine()
+gate = VP.VocabParallelGate(B=B, V_small=V, V_large=V, H_small=Hd, H_large=8, w=5, d_min=10, tau=1.0,
+                            W_small=VP.shard_of(W, world, rank), W_large=VP.shard_of(Wl, world, rank),
+                            rank=rank, world=world, engine=eng, device=torch.device("cpu"))
+try:
+    gate.run(1, h, torch.zeros((T, B, 8)))
+    raise SystemExit("run() before connect() must be refused")
+except RuntimeError:
+    pass
+nbytes = eng.ead_shard_exchange_bytes(B, world)
+own = np.memmap(os.path.join(TMP, f"xchg_{{rank}}.bin"), dtype=np.float32, mode="w+", shape=(nbytes // 4,))
+own[:] = 0
+own.flush()
+dist.barrier()                                              # every buffer exists and is clear
+bufs = [own if r == rank else np.memmap(os.path.join(TMP, f"xchg_{{r}}.bin"), dtype=np.float32, mode="r+",
+                                        shape=(nbytes // 4,)) for r in range(world)]
+gate.connect(bufs)
+assert eng.shard == rank and eng.connected_to[rank] is own
+tok = torch.zeros((T, B), dtype=torch.int32); H = torch.zeros((T, B), dtype=torch.float32)
+gate.run(T - 1, h, torch.zeros((T, B, 8)), tok, H)
+gate.step(h[T - 1], torch.zeros((B, 8)), tok[T - 1], H[T - 1])   # a connected step is one call as well
+for t in range(T):
+    z = h[t].double().numpy() @ W.double().numpy().T
+    for b in range(B):
+        assert abs(float(H[t, b]) - O.entropy(z[b])) < 1e-6, (t, b)
+        assert int(tok[t, b]) == O.greedy(z[b])[0]
+# what the last two steps left in this rank's buffer: source r's arg max lies in slice r
+ints = own.reshape(2, world, B, 8).view(np.int32)
+for r in range(world):
+    b0, e0 = VP.shard_rows(V, world, r)
+    assert ((ints[:, r, :, 3] >= b0) & (ints[:, r, :, 3] < e0)).all()
+assert sorted(ints[:, :, :, 7].reshape(2, -1)[:, 0].tolist()) == [T - 1, T]
+dist.barrier()
+dist.destroy_process_group()
+print("rank", rank, "ok")
+"""
+
+
+def test_vocab_parallel_connected_route_over_two_gloo_ranks(tmp_path):
+    script = tmp_path / "vp_connected_worker.py"
+    script.write_text(_VP_CONNECTED_WORKER.format(root=ROOT, tmp=str(tmp_path)))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+           "--master-addr", "127.0.0.1", "--master-port", "29635", str(script)]
+    res = subprocess.run(cmd, capture_output=True, text=True, timeout=240)
+    assert res.returncode == 0, res.stdout + res.stderr
+    assert res.stdout.count("ok") == 2
+
+
+def test_connect_symmetric_against_a_stand_in_for_symmetric_memory():
+    """`connect_symmetric` in the order that keeps it safe: allocate, rendezvous over the right
+    group, clear the buffer, barrier (nobody stores before everybody has cleared), and only then
+    hand the peers' addresses to the library, in rank order."""
+    import torch
+    from paper_2502_06833_b200 import binding, vocab_parallel as VP
+
+    log = []
+
+    class Engine:
+        EAD_SHARD_RECORD_BYTES = 32
+        ead_shard_range = staticmethod(binding.ead_shard_range)
+
+        def ead_shard_exchange_bytes(self, B, n):
+            return 2 * n * B * 32
+
+        def ead_create(self, **kw):
+            return 1
+
+        def ead_shard_connect(self, ctx, shard, exchange):
+            log.append(("connect", shard, list(exchange), bool((buffers[0] == 0).all())))
+
+        def ead_destroy(self, ctx):
+            pass
+
+    buffers = []
+
+    class Handle:
+        buffer_ptrs = [0x1000, 0x2000, 0x3000]
+
+    class Symm:
+        @staticmethod
+        def empty(n, dtype, device):
+            log.append(("empty", n, dtype, str(device)))
+            buffers.append(torch.full((n,), 255, dtype=dtype))
+            return buffers[-1]
+
+        @staticmethod
+        def rendezvous(buf, group):
+            log.append(("rendezvous", buf is buffers[-1], group))
+            return Handle
+
+    class Dist:
+        class group:
+            WORLD = "world-group"
+
+        @staticmethod
+        def barrier(group=None):
+            log.append(("barrier", group, bool((buffers[0] == 0).all())))
+
+    W = torch.zeros((384, 8))
+    gate = VP.VocabParallelGate(B=4, V_small=1100, V_large=1100, H_small=8, H_large=8, w=5, d_min=10, tau=1.0,
+                                W_small=W[:384], W_large=W[:384], rank=1, world=3, group="sub-group",
+                                engine=Engine(), dist=Dist, device=torch.device("cpu"))
+    gate.connect_symmetric(symm=Symm)
+    assert [e[0] for e in log] == ["empty", "rendezvous", "barrier", "connect"]
+    assert log[0][1] == 2 * 3 * 4 * 32 and log[0][2] == torch.uint8
+    assert log[1] == ("rendezvous", True, "sub-group")
+    assert log[2] == ("barrier", "sub-group", True)                 # cleared before the barrier
+    assert log[3] == ("connect", 1, [0x1000, 0x2000, 0x3000], True)
+    assert gate.connected
+    log.clear()
+    gate2 = VP.VocabParallelGate(B=4, V_small=1100, V_large=1100, H_small=8, H_large=8, w=5, d_min=10, tau=1.0,
+                                 W_small=W[:384], W_large=W[:384], rank=0, world=3, engine=Engine(), dist=Dist,
+                                 device=torch.device("cpu"))
+    gate2.connect_symmetric(symm=Symm)
+    assert log[1][2] == "world-group" and log[2][1] is None         # default group
