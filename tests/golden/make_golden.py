@@ -30,12 +30,18 @@ PLANS = {
     "llama_b1_switching": (configs.LLAMA_B1_SWITCHING, {}, 0, [0], 2048),
     "llama_b64": (configs.LLAMA_B64, {}, 12, [0, 9, 18, 27, 36, 45, 54, 63], 1024),
     "qwen_b256": (configs.QWEN_B256, {}, 12, [0, 85, 170, 255], 512),
-    "qwen_b1024_f0": (configs.STRESS_0, {}, 2, [0, 1023], 64),
+    "qwen_b1024_f0": (configs.STRESS_0, {}, 2, [0, 1023], 256),
     "qwen_b1024_f25": (configs.STRESS_25, {}, 12, [0, 341, 682, 1023], 256),
     "qwen_b1024_f50": (configs.STRESS_50, {}, 0, [0, 146, 292, 438, 584, 730, 876, 1023], 256),
-    "qwen_b1024_f100": (configs.STRESS_100, {}, 2, [0, 1023], 64),
-    "qwen_b1024_w1": (configs.STRESS_50, dict(w=1, d_min=1), 0, [0, 511, 1023], 96),
-    "qwen_b1024_w20": (configs.STRESS_50, dict(w=20, d_min=10), 0, [0, 511, 1023], 96),
+    "qwen_b1024_f100": (configs.STRESS_100, {}, 2, [0, 1023], 256),
+    "qwen_b1024_w1": (configs.STRESS_50, dict(w=1, d_min=1), 0, [0, 511, 1023], 256),
+    "qwen_b1024_w20": (configs.STRESS_50, dict(w=20, d_min=10), 0, [0, 511, 1023], 256),
+    # window and dwell sweep on the 25 % mix ((w, d_min) = (5, 10) is qwen_b1024_f25 itself)
+    "qwen_b1024_f25_w1_d1": (configs.STRESS_25, dict(w=1, d_min=1), 0, [0, 511, 1023], 256),
+    "qwen_b1024_f25_w1_d10": (configs.STRESS_25, dict(w=1, d_min=10), 0, [0, 511, 1023], 256),
+    "qwen_b1024_f25_w5_d1": (configs.STRESS_25, dict(w=5, d_min=1), 0, [0, 511, 1023], 256),
+    "qwen_b1024_f25_w20_d1": (configs.STRESS_25, dict(w=20, d_min=1), 0, [0, 511, 1023], 256),
+    "qwen_b1024_f25_w20_d10": (configs.STRESS_25, dict(w=20, d_min=10), 0, [0, 511, 1023], 256),
 }
 
 
