@@ -46,16 +46,14 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, SmemCtrl
 {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
-    uint32_t spins = 0;
     for (;;) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 0x3FFu) == 0) {
-            if (*reinterpret_cast<volatile uint32_t *>(&c->abort)) return false;
-            if (globaltimer_ns() - t0 > kWaitLimitNs) {
-                *reinterpret_cast<volatile uint32_t *>(&c->abort) = 1u;
-                atomicOr(&ctl->status, kStatusWaitExpired);
-                return false;
-            }
+        // suspended until the phase completes or 4 us have passed: no polling in between
+        if (mbar_try_wait_hint(bar, parity, 4000u)) return true;
+        if (*reinterpret_cast<volatile uint32_t *>(&c->abort)) return false;
+        if (globaltimer_ns() - t0 > kWaitLimitNs) {
+            *reinterpret_cast<volatile uint32_t *>(&c->abort) = 1u;
+            atomicOr(&ctl->status, kStatusWaitExpired);
+            return false;
         }
     }
 }

@@ -64,6 +64,23 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok;
 }
 
+// As mbar_try_wait, but the thread may stay suspended for up to `hint_ns` before the instruction
+// returns (the hardware wakes it when the phase completes): a waiting warp then issues next to
+// nothing.  That matters on the SM sub-partition that also hosts the MMA-issuing warp: every
+// instruction another warp issues there delays the tensor pipe's instruction stream.
+__device__ __forceinline__ uint32_t mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t hint_ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok;
+}
+
 // ----------------------------------------------------------------- TMA
 __device__ __forceinline__ uint64_t l2_policy_evict_first()
 {
