@@ -22,8 +22,8 @@ at least 32 warm-up steps (so that the mix of heads is the configuration's, not 
 Algorithm 1's first d_min tokens) and at least 32 timed steps per repeat.  `--config NAME`
 measures that configuration alone.
 
-With N > 1 every rank runs an independent replica of the workload (the path has no
-cross-sequence term and is not sharded).  `--impl reference` times the CPU oracle alone
+With N > 1 every rank runs an independent replica of the headline workload (the path has no
+cross-sequence term and is not sharded); `per_config` is reported by single-GPU runs only.  `--impl reference` times the CPU oracle alone
 (there is no reference implementation of this path): rank 0 only, a bounded number of steps.
 """
 from __future__ import annotations
@@ -465,7 +465,8 @@ def per_config_entry(m: dict) -> dict:
 
 def run_ours(args):
     rt = Runtime()
-    everything = args.config in (None, "all")
+    # the per-configuration list is a single-GPU report: with N > 1 every rank would only repeat it
+    everything = args.config in (None, "all") and rt.world == 1
     head_cfg = configs.ALL[HEADLINE if everything else args.config]
     W = max(3, args.warmup)
     K = args.steps if args.steps is not None else max(1, head_cfg.T - W)

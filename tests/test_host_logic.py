@@ -104,6 +104,56 @@ def test_work_split_of_an_empty_head(E):
     assert s["active"] == 0 and s["col_begin"] == s["col_end"]
 
 
+def test_bench_roofline_picks_the_binding_bound_and_states_both_tensor_fractions():
+    sys.path.insert(0, ROOT)
+    import bench
+    peaks = {"hbm_gbs": 6000.0, "bf16_tflops": 1600.0, "bf16_tflops_sustained": 1200.0, "source": "measured"}
+    # 1.2 GB and 1.2 GFLOP in 250 us: 200 us of HBM time against 1 us of tensor time -> HBM bound
+    r = bench.roofline_of(1.2e9, 1.2e9, 250e-6, 300e-6, peaks)
+    assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["frac_of_burst"] is None
+    assert r["achieved"] == pytest.approx(4800.0) and r["frac"] == pytest.approx(0.8)
+    assert r["step_frac"] == pytest.approx(1.2e9 / 300e-6 / 1e9 / 6000.0)
+    assert r["bound_us"]["hbm"] == pytest.approx(200.0) and r["bound_us"]["tensor_sustained"] == pytest.approx(1.0)
+    # 0.5 GB and 1.2 TFLOP in 1.25 ms: 83 us against 1000 us -> tensor bound, both fractions
+    r = bench.roofline_of(0.5e9, 1.2e12, 1.25e-3, 1.5e-3, peaks)
+    assert r["bound"] == "tensor" and r["peak"] == 1200.0 and r["peak_burst"] == 1600.0
+    assert r["frac"] == pytest.approx(0.8) and r["frac_of_burst"] == pytest.approx(0.6)
+    assert r["step_frac"] == pytest.approx(1.2e12 / 1.5e-3 / 1e12 / 1200.0)
+    assert r["frac"] == pytest.approx(r["achieved"] / r["peak"])
+
+
+def test_bench_ncu_traffic_follows_the_heads_that_were_live():
+    sys.path.insert(0, ROOT)
+    import bench
+    from workloads import configs
+    tab = bench.NCU_DRAM_BYTES_PER_LAUNCH
+    cfg = configs.LLAMA_B1
+    used = np.array([[0]] * 5 + [[1]] * 15, dtype=np.uint8)           # 25 % small-head steps, 75 % large
+    got, files = bench.ncu_traffic(cfg, used)
+    want = 0.25 * tab[("llama_b1", "small")][0] + 0.75 * tab[("llama_b1", "large")][0]
+    assert got == pytest.approx(want) and len(files) == 2 and all(f.startswith("profiles/") for f in files)
+    for f in files:
+        assert os.path.exists(os.path.join(ROOT, f)), f
+    cfg = configs.STRESS_25
+    used = np.zeros((4, cfg.B), dtype=np.uint8)
+    used[:, :300] = 1                                                   # both heads live in every step
+    got, files = bench.ncu_traffic(cfg, used)
+    assert got == pytest.approx(tab[("qwen_b1024", "both")][0])
+    used[:] = 1
+    assert bench.ncu_traffic(cfg, used)[0] == pytest.approx(tab[("qwen_b1024", "large")][0])
+    assert bench.ncu_traffic(configs.TINY, np.zeros((2, 4), dtype=np.uint8)) == (None, None)   # never captured
+
+
+def test_bench_arms_describe_the_workload_with_the_same_keys():
+    sys.path.insert(0, ROOT)
+    import bench
+    from workloads import configs
+    keys = set(bench.config_keys(configs.LLAMA_B1))
+    assert keys == {"workload", "B", "V", "H_small", "H_large", "w", "d_min", "tau"}
+    src = open(os.path.join(ROOT, "bench.py")).read()
+    assert src.count('"config": config_keys(') == 2                     # the reference arm and ours
+
+
 def test_bench_step_costs():
     sys.path.insert(0, ROOT)
     import bench
