@@ -94,7 +94,7 @@ struct ead_ctx {
     uint16_t *hc[2] = {nullptr, nullptr};
     ShardLink *link = nullptr;             // vocabulary-sharded contexts: where the records go (device)
     bool connected = false;                // ead_shard_connect has filled `link`
-    CUtensorMap tmA[2], tmW[2], tmT[2], tmP[2];   // hidden rows; W boxes of 256|128, 16 and 32 rows
+    CUtensorMap tmA[2], tmH[2], tmW[2], tmT[2], tmP[2];   // hidden rows (boxes of a_rows and of 64 rows); W boxes of 256|128, 16 and 32 rows
     cudaGraphExec_t g_one = nullptr, g_chunk = nullptr;
     int64_t launches = 0;
     // staging of ead_run_host (allocated on first use)
@@ -227,10 +227,11 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr, int shar
                              x->tmA[1], x->tmW[0], x->tmW[1], x->tmP[0], x->tmP[1], lp)
     switch (x->small_cols) {
         case 0:
+            lp.half_blocks = 1;
             e = lp.sampling ? launch(ead_lmhead_kernel<true>, lgrid, lblock, x->smem_bytes, s, pdl, x->tmA[0], x->tmA[1],
-                                     x->tmW[0], x->tmW[1], x->tmT[0], x->tmT[1], lp)
+                                     x->tmW[0], x->tmW[1], x->tmT[0], x->tmT[1], x->tmH[0], x->tmH[1], lp)
                             : launch(ead_lmhead_kernel<false>, lgrid, lblock, x->smem_bytes, s, pdl, x->tmA[0], x->tmA[1],
-                                     x->tmW[0], x->tmW[1], x->tmT[0], x->tmT[1], lp);
+                                     x->tmW[0], x->tmW[1], x->tmT[0], x->tmT[1], x->tmH[0], x->tmH[1], lp);
             break;
         case 1: EAD_LAUNCH_SMALL(1); break;
         case 2: EAD_LAUNCH_SMALL(2); break;
@@ -505,6 +506,7 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
         const uint32_t wbox = static_cast<uint32_t>(
             std::min(x->small_cols ? kSmallTileRows : kTileN, (Vm[m] + kUnit - 1) / kUnit * kUnit));
         if (!encode_bf16_2d(&x->tmA[m], x->hc[m], Bpad, Hm[m], x->a_rows) ||
+            !encode_bf16_2d(&x->tmH[m], x->hc[m], Bpad, Hm[m], std::min(x->a_rows, kTileM / 2)) ||
             !encode_bf16_2d(&x->tmW[m], x->W[m], Vm[m], Hm[m], wbox) ||
             !encode_bf16_2d(&x->tmT[m], x->W[m], Vm[m], Hm[m], kUnit) ||
             !encode_bf16_2d(&x->tmP[m], x->W[m], Vm[m], Hm[m], kSmallSegRows))
@@ -1075,7 +1077,7 @@ extern "C" int ead_head_entropy_static(const void *W, const void *h, int32_t B, 
     lp.part_s = sc->part_s;
     lp.part_t = sc->part_t;
     lp.part_i = sc->part_i;
-    ead_lmhead_kernel<false><<<G, kLmheadThreads, smem_bytes, s>>>(tmA, tmA, tmW, tmW, tmT, tmT, lp);
+    ead_lmhead_kernel<false><<<G, kLmheadThreads, smem_bytes, s>>>(tmA, tmA, tmW, tmW, tmT, tmT, tmA, tmA, lp);
     const int rows_per_block = kGateThreads / 32;
     ead_static_merge_kernel<<<(B + rows_per_block - 1) / rows_per_block, kGateThreads, 0, s>>>(sc, B, G, tok, H_out,
                                                                                              status);

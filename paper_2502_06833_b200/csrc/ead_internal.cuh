@@ -164,14 +164,17 @@ __device__ __forceinline__ float lg2_approx(float x)
 }
 
 // Standard Gumbel variate from one random word: u = (2k + 1) / 2^24 with k its top 23 bits
-// (exact in float32, never 0 or 1), g = -ln(-ln u), both logarithms through the hardware
-// base-2 logarithm (absolute error about 2^-22 each: the perturbed logits move by ~1e-6,
+// (exact in float32, never 0 or 1), g = -ln(-ln u).  The inner logarithm is the accurate one:
+// the draw is decided by the largest g, i.e. by u next to 1, where -ln u is about 1 - u and a
+// logarithm with a fixed absolute error (lg2.approx: 2^-22) would be off by percents (seen on
+// a 128 K vocabulary: largest g about 11.8, error 0.02).  The outer one only needs absolute
+// accuracy and goes through the hardware base-2 logarithm (the perturbed logits move by ~1e-6,
 // three orders of magnitude below the gap under which a different draw counts as a near-tie).
 __device__ __forceinline__ float gumbel_from_word(uint32_t word)
 {
     constexpr float kLn2 = 0.69314718055994531f;
     const float u = static_cast<float>(2u * (word >> 9) + 1u) * 5.9604644775390625e-8f;   // 2^-24
-    const float neg_ln_u = -kLn2 * lg2_approx(u);          // in [6e-8, 16.7]
+    const float neg_ln_u = -logf(u);                        // in [6e-8, 16.7], relative error ~1e-7
     return -kLn2 * lg2_approx(neg_ln_u);
 }
 #endif  // __CUDACC__
@@ -199,6 +202,7 @@ struct LmheadParams {
     const int32_t *perm;   // compacted row -> caller's row (the random stream is per caller row)
     uint32_t ctr_off[2];   // vocabulary-sharded use: first row of this slice in the full head, / 4
     int32_t prefetch_boxes;  // small-batch kernel: 16 KiB weight boxes brought into L2 before the dependency wait
+    int32_t half_blocks;     // large-batch kernel: row blocks of at most 64 rows run as M = 64 tiles
 };
 
 }  // namespace ead

@@ -145,12 +145,21 @@ __device__ __forceinline__ void draw_absorb32(Draw &dr, const float (&v)[32], in
     }
 }
 
+// Whether a row block with `rows` real rows is multiplied as an M = 64 tile.  The instruction
+// takes as long as the M = 128 one, but it reads half the hidden rows (so only 64 are brought in)
+// and switches half the multipliers, which under the power cap is what a padded block costs.
+__device__ __forceinline__ bool half_block(const LmheadParams &p, int rows)
+{
+    return p.half_blocks && rows <= kTileM / 2;
+}
+
 // SAMPLE: also track the arg max of z / T + Gumbel noise (temperature sampling).
 template <bool SAMPLE>
 __global__ void __launch_bounds__(kLmheadThreads, 1)
 ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
                   const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
                   const __grid_constant__ CUtensorMap tmT0, const __grid_constant__ CUtensorMap tmT1,
+                  const __grid_constant__ CUtensorMap tmH0, const __grid_constant__ CUtensorMap tmH1,
                   const LmheadParams p)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -185,6 +194,7 @@ ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
         tma_prefetch_desc(&tmA0); tma_prefetch_desc(&tmA1);
         tma_prefetch_desc(&tmW0); tma_prefetch_desc(&tmW1);
         tma_prefetch_desc(&tmT0); tma_prefetch_desc(&tmT1);
+        tma_prefetch_desc(&tmH0); tma_prefetch_desc(&tmH1);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&ctrl->tmem_base), 2 * kTileN);
@@ -214,12 +224,16 @@ ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
                 const CUtensorMap *tA = m ? &tmA1 : &tmA0;
                 const CUtensorMap *tW = m ? &tmW1 : &tmW0;
                 const CUtensorMap *tT = m ? &tmT1 : &tmT0;
+                // a row block of at most 64 rows is multiplied as an M = 64 tile: half the hidden box
+                const bool half = half_block(p, n_rows[m] - sp.rb * kTileM);
+                if (half) tA = m ? &tmH1 : &tmH0;
+                const uint32_t a_tx = half ? a_bytes / 2 : a_bytes;
                 // a weight tile shared by several row blocks should stay in L2 for them
                 const uint64_t pol_w = (sp.R == 1) ? pol_stream : pol_keep;
                 const int kblocks = (p.H[m] + kBlockK - 1) / kBlockK;
                 for (int col0 = sp.col_begin; col0 < sp.col_end && ok; col0 += kTileN) {
                     const int ncols = min(kTileN, sp.col_end - col0);
-                    const uint32_t tx = a_bytes + static_cast<uint32_t>(ncols) * (kBlockK * 2);
+                    const uint32_t tx = a_tx + static_cast<uint32_t>(ncols) * (kBlockK * 2);
                     for (int kb = 0; kb < kblocks; ++kb, ++it) {
                         const uint32_t s = it % stages;
                         const uint32_t ph = (it / stages) & 1u;
@@ -262,7 +276,9 @@ ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
                         break;
                     }
                     tc_fence_after_sync();
-                    const uint32_t idesc = umma_idesc_bf16_m128(static_cast<uint32_t>(ncols));
+                    const uint32_t idesc = half_block(p, n_rows[m] - sp.rb * kTileM)
+                                               ? umma_idesc_bf16_m64(static_cast<uint32_t>(ncols))
+                                               : umma_idesc_bf16_m128(static_cast<uint32_t>(ncols));
                     const uint32_t d_tmem = tmem_base + buf * kTileN;
                     for (int kb = 0; kb < kblocks; ++kb, ++it) {
                         const uint32_t s = it % stages;
@@ -289,14 +305,18 @@ ead_lmhead_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
     } else {
         // ------------------------------------------------------------- epilogue
         const int quad = warp & 3;                   // TMEM lane quadrant this warp may read
-        const int row_in_block = quad * 32 + lane;
         uint32_t tc = 0;
         bool ok = true;
         for (int m = 0; m < 2 && ok; ++m) {
             const HeadSplit sp = split_head(cta, G, n_rows[m], p.V[m]);
             if (!sp.active) continue;
             const int rows_valid = min(kTileM, n_rows[m] - sp.rb * kTileM);
-            const bool warp_has_rows = quad * 32 < rows_valid;
+            // An M = 128 accumulator keeps row r of the block in TMEM lane r; an M = 64 one keeps
+            // its 64 rows in the lower 16 lanes of each 32-lane quadrant (row r in lane
+            // (r / 16) * 32 + r % 16), the upper 16 lanes hold nothing.
+            const bool half = half_block(p, rows_valid);
+            const int row_in_block = half ? (lane < 16 ? quad * 16 + lane : kTileM) : quad * 32 + lane;
+            const bool warp_has_rows = (half ? quad * 16 : quad * 32) < rows_valid;
             RowStat st;
             rowstat_reset(st);
             // sampling: this thread's sequence draws from its own stream (caller's row, step)

@@ -212,6 +212,13 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr)
     return (static_cast<uint64_t>(hi) << 32) | lo;
 }
 
+// The same with M = 64 (N a multiple of 8): the accumulator then occupies lanes 0-15 of each
+// 32-lane quadrant of TMEM.
+__device__ __forceinline__ uint32_t umma_idesc_bf16_m64(uint32_t n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((64u >> 4) << 24);
+}
+
 // Instruction descriptor of kind::f16 with bf16 A and B (both K-major), fp32 D,
 // M = 128 and N = n (multiple of 16, 16..256).
 __device__ __forceinline__ uint32_t umma_idesc_bf16_m128(uint32_t n)

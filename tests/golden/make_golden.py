@@ -42,16 +42,28 @@ PLANS = {
     "qwen_b1024_f25_w5_d1": (configs.STRESS_25, dict(w=5, d_min=1), 0, [0, 511, 1023], 256),
     "qwen_b1024_f25_w20_d1": (configs.STRESS_25, dict(w=20, d_min=1), 0, [0, 511, 1023], 256),
     "qwen_b1024_f25_w20_d10": (configs.STRESS_25, dict(w=20, d_min=10), 0, [0, 511, 1023], 256),
+    # Algorithm 1's sampling lines at the benchmark shapes (temperature and seed in SAMPLING)
+    "llama_b1_sampled": (configs.LLAMA_B1_SWITCHING, {}, 0, [0], 256),
+    "llama_b64_sampled": (configs.LLAMA_B64, {}, 2, [5, 58], 96),
+    "qwen_b1024_f50_sampled": (configs.STRESS_50, {}, 0, [3, 700], 64),
+}
+
+# name -> (temperature, seed of the random stream); every other plan is greedy
+SAMPLING = {
+    "llama_b1_sampled": (0.8, 0x5EED0001),
+    "llama_b64_sampled": (1.0, 0x5EED0002),
+    "qwen_b1024_f50_sampled": (1.3, 0x5EED0003),
 }
 
 
 def make(name: str) -> None:
     cfg, over, T_head, rows, T = PLANS[name]
     cfg = cfg.with_(**over)
+    temperature, rng_seed = SAMPLING.get(name, (0.0, 0))
     t0 = time.time()
     wl = synth.Workload(cfg, T=T)
     kw = dict(w=cfg.w, d_min=cfg.d_min, tau=float(np.float32(cfg.tau)), unit=cfg.unit,
-              start_model=cfg.start_model)
+              start_model=cfg.start_model, temperature=temperature, seed=rng_seed)
     out = {}
     if T_head:
         o = O.run(wl.W_small, wl.W_large, wl.h_small, wl.h_large, T=T_head, **kw)
@@ -60,7 +72,8 @@ def make(name: str) -> None:
     out.update({"rows_" + k: v for k, v in o.items()})
     meta = dict(B=cfg.B, T=T, V=cfg.V, H_small=cfg.H_small, H_large=cfg.H_large, w=cfg.w,
                 d_min=cfg.d_min, tau=float(np.float32(cfg.tau)), unit=cfg.unit,
-                start_model=cfg.start_model, seed=cfg.seed, T_head=T_head)
+                start_model=cfg.start_model, seed=cfg.seed, T_head=T_head, temperature=temperature,
+                rng_seed=rng_seed)
     np.savez_compressed(os.path.join(HERE, f"oracle_{name}.npz"),
                         meta=np.array(repr(meta)), **out)
     cells = T_head * cfg.B + len(rows) * T

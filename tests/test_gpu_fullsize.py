@@ -24,10 +24,10 @@ def _plans():
     spec = importlib.util.spec_from_file_location("make_golden", os.path.join(GOLDEN, "make_golden.py"))
     mod = importlib.util.module_from_spec(spec)
     spec.loader.exec_module(mod)
-    return mod.PLANS
+    return mod.PLANS, mod.SAMPLING
 
 
-PLANS = _plans()
+PLANS, SAMPLING = _plans()
 
 
 @functools.lru_cache(maxsize=2)
@@ -59,7 +59,9 @@ def test_full_size_against_stored_oracle(name):
 
     wl = _hidden(_chain_key(cfg), T)
     Ws, Wl = _head(cfg.seed, 0, cfg.V, cfg.H_small), _head(cfg.seed, 1, cfg.V, cfg.H_large)
-    with GpuGate(cfg, Ws, Wl) as g:
+    temperature, rng_seed = SAMPLING.get(name, (0.0, 0))
+    assert meta.get("temperature", 0.0) == temperature and meta.get("rng_seed", 0) == rng_seed
+    with GpuGate(cfg, Ws, Wl, temperature=temperature, seed=rng_seed) as g:
         info = g.E.ead_launch_info(g.ctx)
         out = g.run(wl.h_small, wl.h_large, "run")
     assert info["ctas"] >= 100
