@@ -67,11 +67,11 @@ NCU_DRAM_BYTES_PER_LAUNCH = {
     ("llama_b1", "large"): (1.05726e9, "profiles/lmhead_small_kernel_llama_b1_ncu_full.md"),
     ("llama_b1", "small"): (5.3285e8, "profiles/lmhead_kernels_other_configs_ncu_counters.md"),
     ("llama_b64", "both"): (1.5823e9, "profiles/lmhead_small_kernel_llama_b64_ncu_full.md"),
-    ("qwen_b256", "both"): (2.0374e9, "profiles/lmhead_kernel_qwen_b256_ncu_counters.md"),
-    ("qwen_b1024", "small"): (4.7419e8, "profiles/lmhead_kernels_other_configs_ncu_counters.md"),
-    # captured at 25 % and 50 % of the rows on the large head (2.0679 and 2.0830 GB): their mean
-    ("qwen_b1024", "both"): (2.0755e9, "profiles/lmhead_kernels_other_configs_ncu_counters.md"),
-    ("qwen_b1024", "large"): (1.5878e9, "profiles/lmhead_kernel_qwen_b1024_all_large_ncu_full.md"),
+    ("qwen_b256", "both"): (2.0384e9, "profiles/lmhead_kernel_qwen_b256_ncu_counters.md"),
+    ("qwen_b1024", "small"): (4.7385e8, "profiles/lmhead_kernels_other_configs_ncu_counters.md"),
+    # captured at 25 % and 50 % of the rows on the large head (2.0677 and 2.0622 GB): their mean
+    ("qwen_b1024", "both"): (2.0649e9, "profiles/lmhead_kernels_other_configs_ncu_counters.md"),
+    ("qwen_b1024", "large"): (1.6049e9, "profiles/lmhead_kernel_qwen_b1024_all_large_ncu_full.md"),
 }
 
 
