@@ -164,17 +164,21 @@ __device__ __forceinline__ float lg2_approx(float x)
 }
 
 // Standard Gumbel variate from one random word: u = (2k + 1) / 2^24 with k its top 23 bits
-// (exact in float32, never 0 or 1), g = -ln(-ln u).  The inner logarithm is the accurate one:
-// the draw is decided by the largest g, i.e. by u next to 1, where -ln u is about 1 - u and a
-// logarithm with a fixed absolute error (lg2.approx: 2^-22) would be off by percents (seen on
-// a 128 K vocabulary: largest g about 11.8, error 0.02).  The outer one only needs absolute
-// accuracy and goes through the hardware base-2 logarithm (the perturbed logits move by ~1e-6,
-// three orders of magnitude below the gap under which a different draw counts as a near-tie).
+// (exact in float32, never 0 or 1), g = -ln(-ln u).  The draw is decided by the largest g, i.e.
+// by u next to 1, where -ln u is about 1 - u: there the hardware base-2 logarithm, whose error
+// is absolute (2^-22), would be off by percents (seen on a 128 K vocabulary: largest g about
+// 11.8, error 0.02, a wrong token).  So -ln u is the series w + w^2/2 + w^3/3 + w^4/4 in
+// w = 1 - u (exact in float32) for w < 1/64 and -ln 2 lg2(u) elsewhere, both within 1e-5
+// relative; the outer logarithm only needs absolute accuracy.  The perturbed logits then move
+// by ~1e-5, two orders of magnitude below the gap under which a different draw counts as a
+// near-tie.
 __device__ __forceinline__ float gumbel_from_word(uint32_t word)
 {
     constexpr float kLn2 = 0.69314718055994531f;
     const float u = static_cast<float>(2u * (word >> 9) + 1u) * 5.9604644775390625e-8f;   // 2^-24
-    const float neg_ln_u = -logf(u);                        // in [6e-8, 16.7], relative error ~1e-7
+    const float w = 1.0f - u;
+    const float series = w * fmaf(w, fmaf(w, fmaf(w, 0.25f, 0.33333334f), 0.5f), 1.0f);
+    const float neg_ln_u = w < 0.015625f ? series : -kLn2 * lg2_approx(u);   // in [6e-8, 16.7]
     return -kLn2 * lg2_approx(neg_ln_u);
 }
 #endif  // __CUDACC__
