@@ -238,8 +238,10 @@ def oracle_sample(cfg, wl, budget_s: float, max_steps: int, skip: int):
 
     skip = min(skip, wl.T - 1)
     t_skip, _ = timed(skip)
-    t_probe, _ = timed(skip + 1)
+    t_probe, probe = timed(skip + 1)
     per_step = max(t_probe - t_skip, t_skip / max(skip, 1), 1e-4)
+    if float(probe["used"][skip].mean()) < 0.5:            # probed on the small head: later steps may cost
+        per_step *= max(1.0, cfg.H_large / cfg.H_small)    # as much as the large one
     n = int(max(1, min(max_steps, wl.T - skip, (budget_s - t_skip) / per_step)))
     t_all, out = timed(skip + n)
     dt = max(t_all - t_skip, 1e-9)
@@ -476,7 +478,12 @@ def run_ours(args):
     cpu = None
     if rt.rank == 0 and rt.world == 1 and not args.no_cpu_baseline:
         budget = float(args.cpu_seconds if args.cpu_seconds is not None else 15.0)
-        rate, n, dt, cores, fl = oracle_sample(head_cfg, head["wl"], budget, K, skip=W)
+        # the sample is sized by the time budget, not by K: a short timed region would otherwise
+        # leave the oracle a fraction of a second (inputs of up to 1 GB for the extra steps)
+        per_step_bytes = 2 * head_cfg.B * (head_cfg.H_small + head_cfg.H_large)
+        T_cpu = int(min(head_cfg.T, max(W + K, W + min(2048, (1 << 30) // per_step_bytes))))
+        wl_cpu = head["wl"] if T_cpu <= W + K else rt.cache.get(head_cfg, T_cpu)
+        rate, n, dt, cores, fl = oracle_sample(head_cfg, wl_cpu, budget, T_cpu - W, skip=W)
         cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"steps {W}..{W + n} of the same workload, all {head_cfg.B} rows "
                          f"(large-head share {fl:.2f}), {dt:.1f} s"}
