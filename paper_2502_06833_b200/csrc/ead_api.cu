@@ -736,7 +736,7 @@ int ead_shard_gate(ead_ctx *x, const void *all_records, int32_t n_shards, int32_
     out.next = next_model;
     const GateParams gp = gate_params(x, 0);
     ead_shard_gate_kernel<<<(x->cfg.B + 127) / 128, 128, 0, x->stream>>>(
-        gp, static_cast<const ShardRecord *>(all_records), n_shards, out, all_records ? 1 : 3);
+        gp, static_cast<const ShardRecord *>(all_records), n_shards, out, all_records ? 0 : 1);
     x->launches += 1;
     return cudaGetLastError() == cudaSuccess ? EAD_OK : EAD_ECUDA;
 }

@@ -463,27 +463,26 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_wide_kernel(const
 // all n shards for this step in shard order and finishes the step exactly as the single-GPU
 // merge does.  Every shard runs this on the same records in the same order, so the per-sequence
 // state stays identical on all of them without further communication.
-//   mode 1: `all` = [n][B] records gathered by the caller; outputs `out` are [B]
-//   mode 2: records arrive in this shard's exchange buffer (link->all[self]), stored there by
-//           the merge kernels of all shards; the thread waits for each record's step word
-//           (bounded: a shard that never delivers sets EAD_STATUS_WAIT_EXPIRED); outputs go
-//           to the buffers of the current run (p.args)
-//   mode 3: records as in mode 2, outputs as in mode 1 (the two halves of a step called apart)
+// (Whole steps of a connected context do not come here: there the merge kernels finish the rows
+// themselves.)  Outputs `out` are [B].
+//   from_exchange = 0: `all` = [n][B] records gathered by the caller
+//   from_exchange = 1: records arrive in this shard's exchange buffer (link->all[self]), stored
+//           there by the merge kernels of all shards; the thread waits for each record's step
+//           word (bounded: a shard that never delivers sets EAD_STATUS_WAIT_EXPIRED)
 __global__ void __launch_bounds__(128)
-ead_shard_gate_kernel(const GateParams p, const ShardRecord *all, int n_shards, RunArgs out, int mode)
+ead_shard_gate_kernel(const GateParams p, const ShardRecord *all, int n_shards, RunArgs out, int from_exchange)
 {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     griddep_launch_dependents();
     griddep_wait();                               // this shard's own records, state of the last step
     const int t_step = p.ctl->cur_t;
     const int step1 = p.ctl->cur_x + 1;
-    if (mode >= 2) {
+    if (from_exchange) {
         const ShardLink &lk = *p.link;
         n_shards = lk.n;
         all = lk.all[lk.self] + static_cast<size_t>((step1 - 1) & 1) * lk.n * p.B;
     }
-    if (mode == 2) out = *p.args;
-    else out.run_base = t_step;
+    out.run_base = t_step;
     if (b == 0) {                                 // nobody in this kernel reads step or xstep
         p.ctl->step = t_step + 1;
         p.ctl->xstep = step1;
@@ -503,7 +502,7 @@ ead_shard_gate_kernel(const GateParams p, const ShardRecord *all, int n_shards, 
     Partial acc{kNegSentinel, 0.f, 0.f, 0x7fffffff};
     Draw draw{-INFINITY, 0x7fffffff};
     // one deadline for all of this thread's waits; none at all once a wait has expired before
-    const bool patient = mode >= 2 && !(p.ctl->status & kStatusWaitExpired);
+    const bool patient = from_exchange && !(p.ctl->status & kStatusWaitExpired);
     const bool agree = gather_shard_records(p, all, n_shards, b, model, step1, patient, acc, draw);
     if (!agree) {                                 // a shard is on another step or saw other flags
         atomicOr(&p.ctl->status, kStatusShardMismatch);
