@@ -216,6 +216,41 @@ def test_largest_batch_and_zero_steps():
     compare(out, ora, cfg.tau)
 
 
+@pytest.mark.parametrize("B", [129, 192, 193, 256, 320])
+def test_last_row_block_at_the_half_tile_boundary(B):
+    """Every row on the large head, so its last row block has B - 128 (- 128) rows: 1, 64 and 65
+    rows straddle the switch between the M = 64 and the M = 128 tile; 256 has no short block,
+    320 a 64-row one after two full blocks."""
+    cfg = _cfg(B=B, V=2100, H_small=64, H_large=192, T=6, tau=-1.0, start_model=1, d_min=1)
+    wl = synth.Workload(cfg)
+    ora = _oracle(cfg, wl)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        out = g.run(wl.h_small, wl.h_large, "run")
+        again = g.run(wl.h_small, wl.h_large, "step")
+    log = compare(out, ora, cfg.tau)
+    assert log["cells"] == B * cfg.T and ora["used"].all()
+    assert np.array_equal(out["tok"][-1], again["tok"][-1])
+
+
+def test_a_step_with_every_sequence_ended_computes_nothing_and_keeps_the_state():
+    cfg = _cfg(B=150, V=900, T=6, tau=_mid_tau(900))
+    wl = synth.Workload(cfg)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        g.run(wl.h_small[:3], wl.h_large[:3], "run")
+        before = g.E.ead_get_state(g.ctx)
+        g.E.ead_set_done(g.ctx, np.ones(cfg.B, dtype=np.uint8))
+        out = g.run(wl.h_small[3:], wl.h_large[3:], "run")
+        after = g.E.ead_get_state(g.ctx)
+        assert g.E.ead_status(g.ctx) == 0
+    assert (out["tok"] == -1).all() and np.isnan(out["H"]).all() and np.isnan(out["Hbar"]).all()
+    assert np.array_equal(out["used"], out["next"])
+    pad = (4 - cfg.B % 4) % 4
+    done_at = 16 + cfg.B + pad
+    # everything but the step count and the done mask is as before
+    assert before[16:done_at] == after[16:done_at] and before[done_at + cfg.B + pad:] == after[done_at + cfg.B + pad:]
+    assert after[done_at:done_at + cfg.B] == bytes([1]) * cfg.B
+
+
 def test_maximum_batch_of_the_interface():
     """B = 4096, the largest batch ead_create takes: 32 row blocks over both heads, four or
     five CTAs per row block."""
