@@ -21,6 +21,13 @@
 //   warps 2-5   epilogue: tcgen05.ld 32 columns at a time, online update.
 // Accumulators are double buffered so that the epilogue of one tile overlaps the
 // MMAs of the next.
+//
+// A head's rows come in blocks of 128.  Its last block is usually short: with at most 64
+// rows it is multiplied as an M = 64 tile (a 64-row hidden box; the accumulator then sits in
+// the lower 16 lanes of each 32-lane TMEM quadrant), otherwise as an M = 128 tile whose rows
+// beyond the real ones are zeros (the compaction kernel keeps them so).  Neither saves
+// cycles - the instruction takes 128 cycles whatever M is - but both save power, which is
+// what a run of seconds is bound by.
 #pragma once
 #include "ead_internal.cuh"
 #include "ptx_sm100.cuh"
