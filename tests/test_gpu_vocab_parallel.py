@@ -294,3 +294,56 @@ def test_stepping_calls_need_a_connected_context():
             with pytest.raises(E.EadError) as err:
                 call()
             assert err.value.code == E.EAD_EINVALID_ARG
+
+
+# torch's symmetric memory with a process group of ONE rank on the one GPU there is: the real
+# allocator, rendezvous and pointer table behind `connect_symmetric`, then whole runs through the
+# buffer it returned.  (Several ranks would need several GPUs; kernels of different ranks that
+# wait for one another never share a GPU here.)
+_SYMM_WORKER = r"""
+import os, sys
+sys.path.insert(0, {root!r}); sys.path.insert(0, os.path.join({root!r}, "tests"))
+os.environ["MASTER_ADDR"] = "127.0.0.1"; os.environ["MASTER_PORT"] = "29741"
+import numpy as np, torch, torch.distributed as dist
+torch.cuda.set_device(0)
+dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+from paper_2502_06833_b200 import binding as E, vocab_parallel as VP
+from oracle import ead_oracle as O
+from workloads import synth
+from workloads.configs import EADConfig
+from gpu_util import compare, to_dev_bf16
+cfg = EADConfig(name="case", B=5, T=40, H_small=64, H_large=128, V=1500, tau=6.2, w=3, d_min=2, seed=11,
+                stay_easy=0.8, stay_hard=0.8)
+wl = synth.Workload(cfg)
+ora = O.run(wl.W_small, wl.W_large, wl.h_small, wl.h_large, w=cfg.w, d_min=cfg.d_min, tau=float(np.float32(cfg.tau)))
+Ws, Wl = to_dev_bf16(wl.W_small), to_dev_bf16(wl.W_large)
+gate = VP.VocabParallelGate(B=cfg.B, V_small=cfg.V, V_large=cfg.V, H_small=cfg.H_small, H_large=cfg.H_large, w=cfg.w,
+                            d_min=cfg.d_min, tau=cfg.tau, W_small=Ws, W_large=Wl, rank=0, world=1)
+gate.connect_symmetric()
+buf, handle = gate._symm
+assert buf.numel() == E.ead_shard_exchange_bytes(cfg.B, 1) and int(handle.buffer_ptrs[0]) == buf.data_ptr()
+hs, hl = to_dev_bf16(wl.h_small), to_dev_bf16(wl.h_large)
+T, B = cfg.T, cfg.B
+o = dict(tok=torch.zeros((T, B), dtype=torch.int32, device="cuda"), H=torch.zeros((T, B), device="cuda"),
+         Hbar=torch.zeros((T, B), device="cuda"), used=torch.zeros((T, B), dtype=torch.uint8, device="cuda"),
+         next=torch.zeros((T, B), dtype=torch.uint8, device="cuda"))
+gate.run(T, hs, hl, o["tok"], o["H"], o["Hbar"], o["used"], o["next"])
+assert gate.status() == 0
+log = compare({{k: v.cpu().numpy() for k, v in o.items()}}, ora, cfg.tau)
+assert log["cells"] == T * B and 0 < ora["used"].mean() < 1
+assert buf.view(torch.int32).reshape(2, 1, B, 8)[:, 0, :, 7].max().item() == T      # the records went through it
+gate.close()
+dist.destroy_process_group()
+print("symmetric ok")
+"""
+
+
+def test_connect_symmetric_on_real_symmetric_memory_with_one_rank(tmp_path):
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    script = tmp_path / "symm_worker.py"
+    script.write_text(_SYMM_WORKER.format(root=root))
+    res = subprocess.run([sys.executable, str(script)], capture_output=True, text=True, timeout=300)
+    assert res.returncode == 0 and "symmetric ok" in res.stdout, (res.stdout + res.stderr)[-3000:]
