@@ -630,14 +630,17 @@ int ead_run_host(ead_ctx *x, int32_t T, const void *h_small_seq, const void *h_l
     const OutLayout l = out_layout(S, c.B);
     const size_t row_s = static_cast<size_t>(c.B) * c.H_small * 2, row_l = static_cast<size_t>(c.B) * c.H_large * 2;
     const uint8_t *hs = static_cast<const uint8_t *>(h_small_seq), *hl = static_cast<const uint8_t *>(h_large_seq);
-    const int chunks = (T + S - 1) / S;
+    // Chunks grow from 4 steps to the staging size: the first chunk's copy is the one nothing
+    // can hide, so it is kept short; from then on copies run under the computation.
+    int t0 = 0, ramp = 4;
     // A failed call inside the loop must not leave copies to or from the caller's buffers in
     // flight: every error path falls through to the synchronisation below.
 #define EAD_TRY(x)                     \
     if (rc == EAD_OK && (x) != cudaSuccess) rc = EAD_ECUDA
-    for (int k = 0; k < chunks && rc == EAD_OK; ++k) {
+    for (int k = 0; t0 < T && rc == EAD_OK; ++k) {
         const int i = k & 1;
-        const int t0 = k * S, n = std::min(S, T - t0);
+        const int n = std::min(std::min(S, ramp), T - t0);
+        ramp = std::min(S, 2 * ramp);
         const size_t cells = static_cast<size_t>(n) * c.B;
         // inputs of chunk k -> staging buffer i, once the compute that read it (chunk k-2) is done
         if (k >= 2) EAD_TRY(cudaStreamWaitEvent(x->in_stream, x->ev_comp[i], 0));
@@ -664,6 +667,7 @@ int ead_run_host(ead_ctx *x, int32_t T, const void *h_small_seq, const void *h_l
         if (next_model)
             EAD_TRY(cudaMemcpyAsync(next_model + o0, o + l.off_next, cells, cudaMemcpyDeviceToHost, x->out_stream));
         EAD_TRY(cudaEventRecord(x->ev_out[i], x->out_stream));
+        t0 += n;
     }
 #undef EAD_TRY
     // the call is synchronous, also when it fails
