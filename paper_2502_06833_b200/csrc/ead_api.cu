@@ -361,7 +361,10 @@ int ensure_staging(ead_ctx *x)
     if (x->st_steps) return EAD_OK;
     const ead_config &c = x->cfg;
     const size_t per_step = static_cast<size_t>(c.B) * (c.H_small + c.H_large) * 2;
-    int steps = static_cast<int>(std::max<size_t>(1, kHostStageBytes / per_step));
+    // about 64 MB per buffer, but room for one 32-step graph if that takes no more than 512 MB
+    // (large batches: a chunk of single-step replays loses the overlap between the steps)
+    const size_t lo = std::max<size_t>(1, std::min<size_t>(kGraphChunk, (512u << 20) / per_step));
+    int steps = static_cast<int>(std::max<size_t>(lo, kHostStageBytes / per_step));
     steps = std::min(steps, 256);
     if (steps > kGraphChunk) steps -= steps % kGraphChunk;
     EAD_CUDA(cudaStreamCreateWithFlags(&x->in_stream, cudaStreamNonBlocking));
