@@ -289,7 +289,8 @@ int ead_shard_gate(ead_ctx *ctx, const void *all_records, int32_t n_shards, int3
                    float *Hbar, uint8_t *model_used, uint8_t *next_model);
 
 /*
- * DIAGNOSTIC.  How the large-batch LM-head kernel divides one head among its CTAs (host-side replica of the rule
+ * DIAGNOSTIC.  How the one-block LM-head kernel (the one behind ead_head_entropy_static) divides
+ * one head among its CTAs (host-side replica of the rule
  * the kernel applies on the device; pure arithmetic, needs no GPU).  With n rows on a head
  * there are R = ceil(n / 128) row blocks; CTA `cta` of `G` serves row block out[1] and
  * vocabulary columns [out[3], out[4]) (multiples of 16; the end may exceed V by < 16).
@@ -297,6 +298,20 @@ int ead_shard_gate(ead_ctx *ctx, const void *all_records, int32_t n_shards, int3
  * Errors: EAD_EINVALID_ARG.
  */
 int ead_plan_split(int32_t cta, int32_t G, int32_t n_rows, int32_t V, int32_t *out);
+
+/*
+ * DIAGNOSTIC.  The same for the kernel that serves B > 128, whose CTAs work in UNITS of row blocks
+ * (host-side replica of the device rule; needs no GPU).  With two_blocks != 0 (heads with a hidden
+ * size of 3072 and more) a unit is two consecutive 128-row blocks against one weight tile, plus
+ * one unit of the last block alone if the head has an odd number of blocks; otherwise every block
+ * is a unit.  Units get CTAs in proportion to their cost (9 : 5 for two blocks : one); member `slot`
+ * of a unit's `group` CTAs takes the 256-column tiles slot + k * group for k < rounds, then its
+ * piece [tail_col0, tail_col0 + tail_cols) of what the whole rounds leave over (cut evenly in
+ * 16-column units; tail_cols may be 0).
+ *   out  host, int32 [8]: {active, two_blocks, first_row_block, slot, group, rounds, tail_col0, tail_cols}
+ * Errors: EAD_EINVALID_ARG (also: more row blocks than CTAs).
+ */
+int ead_plan_units(int32_t cta, int32_t G, int32_t n_rows, int32_t V, int32_t two_blocks, int32_t *out);
 
 /* Waits for outstanding work and frees everything the context owns.  NULL is allowed. */
 void ead_destroy(ead_ctx *ctx);

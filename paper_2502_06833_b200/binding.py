@@ -32,7 +32,7 @@ EAD_SHARD_MAX = 16
 SYMBOLS = ["ead_create", "ead_step", "ead_run", "ead_run_host", "ead_run_timed", "ead_reset", "ead_status",
            "ead_state_size", "ead_get_state", "ead_set_state", "ead_kernel_launches",
            "ead_launch_info", "ead_destroy", "ead_strerror", "ead_head_entropy_static",
-           "ead_plan_split", "ead_usage", "ead_parameter_ratio", "ead_set_done", "ead_get_done",
+           "ead_plan_split", "ead_plan_units", "ead_usage", "ead_parameter_ratio", "ead_set_done", "ead_get_done",
            "ead_shard_range", "ead_shard_partials", "ead_shard_gate", "ead_shard_connect",
            "ead_shard_exchange_bytes"]
 
@@ -104,6 +104,8 @@ def lib() -> C.CDLL:
         L.ead_parameter_ratio.argtypes = [C.c_uint64, C.c_uint64, C.c_double, C.c_double]
         L.ead_plan_split.restype = C.c_int
         L.ead_plan_split.argtypes = [C.c_int32] * 4 + [C.POINTER(C.c_int32)]
+        L.ead_plan_units.restype = C.c_int
+        L.ead_plan_units.argtypes = [C.c_int32] * 5 + [C.POINTER(C.c_int32)]
         L.ead_shard_range.restype = C.c_int
         L.ead_shard_range.argtypes = [C.c_int32] * 3 + [C.POINTER(C.c_int32)] * 2
         L.ead_shard_exchange_bytes.restype = C.c_size_t
@@ -257,6 +259,13 @@ def ead_plan_split(cta, G, n_rows, V) -> dict:
     a = (C.c_int32 * 6)()
     _check(lib().ead_plan_split(int(cta), int(G), int(n_rows), int(V), a), "ead_plan_split")
     return dict(active=a[0], row_block=a[1], slot=a[2], col_begin=a[3], col_end=a[4], group=a[5])
+
+
+def ead_plan_units(cta, G, n_rows, V, two_blocks=True) -> dict:
+    a = (C.c_int32 * 8)()
+    _check(lib().ead_plan_units(int(cta), int(G), int(n_rows), int(V), int(bool(two_blocks)), a), "ead_plan_units")
+    return dict(active=a[0], two_blocks=a[1], row_block=a[2], slot=a[3], group=a[4], rounds=a[5],
+                tail_col0=a[6], tail_cols=a[7])
 
 
 def ead_shard_range(V, n_shards, shard) -> tuple:

@@ -103,6 +103,117 @@ __host__ __device__ inline HeadSplit split_head(int cta, int G, int n, int V)
     return s;
 }
 
+// How the CTAs of the large-batch kernel (B > 128) divide one head.  With n rows there are
+// R = ceil(n / 128) row blocks.  On a head with `two_blocks` set they are taken two at a time:
+// R / 2 units of two blocks and, if R is odd, one unit of the last block alone; otherwise every
+// block is a unit of its own.  Units get CTAs in proportion to their cost (9 : 5 for two blocks :
+// one) and a unit's g CTAs take the head's 256-column tiles round-robin (member `slot` takes
+// tiles slot, slot + g, ...), so that all units sweep the vocabulary at the same pace and a
+// weight tile fetched for one unit is an L2 hit for the others.
+struct UnitSplit {
+    int active;      // this CTA serves a unit of the head
+    int dual;        // 1: row blocks rb and rb + 1; 0: row block rb alone
+    int rb;
+    int slot, g;     // member index within the unit's group of g CTAs (also the partial slot)
+    int rounds;      // whole rounds of 256-column tiles: member `slot` takes tile slot + k * g in round k
+    int tail_col0, tail_cols;   // what is left after the whole rounds is cut evenly (in 16-column
+                                // units) among the g members: this member's piece (tail_cols may be 0)
+    int n_tiles;     // pieces this member multiplies: rounds + (tail_cols > 0)
+};
+
+// Column range [col0, col0 + ncols) of piece k (0 <= k < n_tiles) of a member; vpad = V rounded up to 16.
+__host__ __device__ inline void unit_piece(const UnitSplit &s, int k, int vpad, int &col0, int &ncols)
+{
+    if (k < s.rounds) {
+        col0 = (s.slot + k * s.g) * kTileN;
+        ncols = vpad - col0 < kTileN ? vpad - col0 : kTileN;
+    } else {
+        col0 = s.tail_col0;
+        ncols = s.tail_cols;
+    }
+}
+
+// Units of a head with n rows (R row blocks): D of two blocks, S of one; CTAs per unit gd and gs,
+// in proportion to what a pipeline stage of the unit costs: measured 1386 cycles for two blocks
+// against 763 for one (18 : 10); a single block of at most 64 rows (an M = 64 tile with half the
+// hidden rows) a little less (9).
+__host__ __device__ inline void unit_groups(int G, int n, int two_blocks, int &D, int &S, int &gd, int &gs)
+{
+    const int R = (n + kTileM - 1) / kTileM;
+    // Units of different kinds walk the vocabulary at different rates and cannot share a weight
+    // tile in L2, so a head with both kinds reads its weights twice (measured: 3.2 GB per launch
+    // against 2.06 GB).  With three row blocks that makes the head HBM-bound, and three single
+    // units, which share every tile, are faster (917 against 961 us per step at 25 % large rows).
+    D = (two_blocks && R != 3) ? R / 2 : 0;
+    S = R - 2 * D;
+    gd = gs = 0;
+    if (R <= 0) return;
+    const int w_single = (n - (R - 1) * kTileM) <= kTileM / 2 ? 9 : 10;
+    if (D > 0) {
+        gd = (18 * G) / (18 * D + w_single * S);
+        if (gd < 1) gd = 1;
+    }
+    if (S > 0) {
+        gs = (G - gd * D) / S;
+        if (gs < 1) {                              // fewer CTAs than units are rejected on the host
+            gs = 1;
+            if (D > 0) gd = (G - S) / D > 0 ? (G - S) / D : 1;
+        }
+    }
+}
+
+__host__ __device__ inline UnitSplit split_units(int cta, int G, int n, int V, int two_blocks)
+{
+    UnitSplit s;
+    s.active = 0; s.dual = 0; s.rb = 0; s.slot = 0; s.g = 0;
+    s.rounds = 0; s.tail_col0 = 0; s.tail_cols = 0; s.n_tiles = 0;
+    if (n <= 0) return s;
+    int D, S, gd, gs;
+    unit_groups(G, n, two_blocks, D, S, gd, gs);
+    if (cta < gd * D) {                            // units interleaved: neighbours in the grid share a slot
+        s.active = 1;
+        s.dual = 1;
+        s.rb = 2 * (cta % D);
+        s.slot = cta / D;
+        s.g = gd;
+    } else if (S > 0 && (cta - gd * D) / S < gs) {
+        const int local = cta - gd * D;
+        s.active = 1;
+        s.rb = 2 * D + local % S;
+        s.slot = local / S;
+        s.g = gs;
+    }
+    if (!s.active) return s;
+    // Whole rounds of full tiles, then the rest of the vocabulary in g even pieces, so that the
+    // members of a unit finish together (with whole tiles only, a unit of 74 CTAs on 594 tiles
+    // would wait a ninth round out for two of its members).
+    const int vpad = (V + kUnit - 1) / kUnit * kUnit;
+    const int tiles = (V + kTileN - 1) / kTileN;
+    s.rounds = tiles / s.g;
+    if (s.rounds * s.g * kTileN > vpad) s.rounds -= 1;       // the last whole round would hold the ragged last tile: deal that round out evenly instead
+    const int rest0 = s.rounds * s.g * kTileN;
+    const int rest = vpad - rest0;                            // < g * 256, a multiple of 16
+    if (rest > 0) {
+        const int units16 = rest / kUnit;
+        const int per = (units16 + s.g - 1) / s.g * kUnit;    // columns per member, a multiple of 16, <= 256
+        const int c0 = rest0 + s.slot * per;
+        if (c0 < vpad) {
+            s.tail_col0 = c0;
+            s.tail_cols = vpad - c0 < per ? vpad - c0 : per;
+        }
+    }
+    s.n_tiles = s.rounds + (s.tail_cols > 0 ? 1 : 0);
+    return s;
+}
+
+// Partial slots that the merge has to fold for compacted row `row` of a head with n rows.
+__host__ __device__ inline int unit_slots_of_row(int G, int n, int row, int two_blocks)
+{
+    int D, S, gd, gs;
+    unit_groups(G, n, two_blocks, D, S, gd, gs);
+    return (row / kTileM) < 2 * D ? gd : gs;
+}
+
 #ifdef __CUDACC__
 struct Partial {
     float m, s, t;
@@ -207,6 +318,8 @@ struct LmheadParams {
     uint32_t ctr_off[2];   // vocabulary-sharded use: first row of this slice in the full head, / 4
     int32_t prefetch_boxes;  // small-batch kernel: 16 KiB weight boxes brought into L2 before the dependency wait
     int32_t half_blocks;     // large-batch kernel: row blocks of at most 64 rows run as M = 64 tiles
+    int32_t two_blocks;      // large-batch kernel: bit m set = head m is served in units of two row blocks
+    int32_t ring_bytes;      // large-batch kernel: bytes of the stage ring (cut into 48 or 64 KiB stages per head)
 };
 
 }  // namespace ead

@@ -145,6 +145,9 @@ ead_compact_kernel(StepCtl *ctl, const RunArgs *args, const uint8_t *flag, const
 struct GateParams {
     int32_t B, V, w, d_min, unit, G, slots_stride;
     int32_t n_slots;           // > 0: partial slots per row as written by the small-batch kernel
+    int32_t units;             // != 0: partials come from the large-batch kernel (units of row blocks);
+                               // bit m of two_blocks set = head m is served in units of two row blocks
+    int32_t two_blocks;
     float tau;
     StepCtl *ctl;
     const RunArgs *args;
@@ -378,9 +381,15 @@ __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const Gate
     const int m = i < n0 ? 0 : 1;
     const int r = m ? i - n0 : i;
     const int n_m = m ? n1 : n0;
-    const int R = (n_m + kTileM - 1) / kTileM;
-    int g = p.G / R;
-    if (g < 1) g = 1;
+    // partial slots of the row: one per member of the group that served its row block
+    int g;
+    if (p.units) {
+        g = unit_slots_of_row(p.G, n_m, r, (p.two_blocks >> m) & 1);
+    } else {
+        const int R = (n_m + kTileM - 1) / kTileM;
+        g = p.G / R;
+        if (g < 1) g = 1;
+    }
 
     // ---- cross-CTA merge, fixed order: each lane folds its slots in ascending
     //      order, then a butterfly over the lanes (no float atomics: deterministic)

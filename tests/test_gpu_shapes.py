@@ -44,7 +44,10 @@ SHAPES = [
     (150, 2000, 64, 128),         # one pair block per head, the second CTA of each pair mostly without rows
     (256, 2500, 128, 64),         # both heads together fill exactly one pair block
     (520, 1500, 64, 64),          # up to three pair blocks on one head, ragged last vocabulary tile
-    (700, 9000, 192, 320),        # full 256-wide tiles for every pair, hidden sizes that are multiples of 64
+    (700, 9000, 192, 320),        # full 256-wide tiles, hidden sizes that are multiples of 64
+    (300, 700, 64, 3072),         # large head long enough for two-block units: one unit of two blocks + a short third
+    (520, 1100, 3072, 3136),      # both heads in two-block units, up to four blocks on a head, ragged last tile
+    (200, 600, 3072, 64),         # the small head in two-block units (one unit: 128 rows + the rest)
     (128, 2048, 64, 64),          # exactly one full row block
     (100, 2300, 128, 64),         # four chunks of sequences in the 17..128 variant, the last ragged
     (17, 700, 64, 128),           # smallest batch of that variant
@@ -216,12 +219,14 @@ def test_largest_batch_and_zero_steps():
     compare(out, ora, cfg.tau)
 
 
+@pytest.mark.parametrize("Hl", [192, 3072])
 @pytest.mark.parametrize("B", [129, 192, 193, 256, 320])
-def test_last_row_block_at_the_half_tile_boundary(B):
+def test_last_row_block_at_the_half_tile_boundary(B, Hl):
     """Every row on the large head, so its last row block has B - 128 (- 128) rows: 1, 64 and 65
     rows straddle the switch between the M = 64 and the M = 128 tile; 256 has no short block,
     320 a 64-row one after two full blocks."""
-    cfg = _cfg(B=B, V=2100, H_small=64, H_large=192, T=6, tau=-1.0, start_model=1, d_min=1)
+    cfg = _cfg(B=B, V=2100 if Hl < 1000 else 700, H_small=64, H_large=Hl, T=6 if Hl < 1000 else 3, tau=-1.0,
+               start_model=1, d_min=1)
     wl = synth.Workload(cfg)
     ora = _oracle(cfg, wl)
     with GpuGate(cfg, wl.W_small, wl.W_large) as g:
@@ -300,7 +305,8 @@ def test_usage_counters_follow_the_trace_and_survive_a_checkpoint():
 
 @pytest.mark.parametrize("B,V,Hs,Hl,temp", [(3, 1000, 64, 128, 1.0), (1, 4100, 256, 512, 0.7),
                                             (12, 2500, 128, 64, 1.5), (40, 3000, 64, 128, 1.0),
-                                            (97, 1100, 64, 128, 1.2), (130, 1700, 64, 64, 0.8)])
+                                            (97, 1100, 64, 128, 1.2), (130, 1700, 64, 64, 0.8),
+                                            (290, 800, 64, 3072, 1.1)])
 def test_temperature_sampling_matches_the_oracle_draws(B, V, Hs, Hl, temp):
     """Algorithm 1's sampling lines: same Philox stream and Gumbel-max rule on both sides, so
     the drawn tokens must be identical (up to logged near-ties of the perturbed values);
