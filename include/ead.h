@@ -302,13 +302,17 @@ int ead_plan_split(int32_t cta, int32_t G, int32_t n_rows, int32_t V, int32_t *o
 /*
  * DIAGNOSTIC.  The same for the kernel that serves B > 128, whose CTAs work in UNITS of row blocks
  * (host-side replica of the device rule; needs no GPU).  With two_blocks != 0 (heads with a hidden
- * size of 3072 and more) a unit is two consecutive 128-row blocks against one weight tile, plus
- * one unit of the last block alone if the head has an odd number of blocks; otherwise every block
- * is a unit.  Units get CTAs in proportion to their cost (9 : 5 for two blocks : one); member `slot`
- * of a unit's `group` CTAs takes the 256-column tiles slot + k * group for k < rounds, then its
- * piece [tail_col0, tail_col0 + tail_cols) of what the whole rounds leave over (cut evenly in
- * 16-column units; tail_cols may be 0).
- *   out  host, int32 [8]: {active, two_blocks, first_row_block, slot, group, rounds, tail_col0, tail_cols}
+ * size of 3072 and more) a unit is two consecutive 128-row blocks against one weight tile.  An odd
+ * last block is a unit of its own.  A head of exactly three row blocks is different: if its last
+ * block has at most 64 rows, the two-block unit takes it along as a thin third block (thin16 =
+ * its rows rounded up to 16) and works on tiles of tile_n = 256 - thin16 columns; otherwise it is
+ * served one block per unit, as is every head with two_blocks == 0.  Units get CTAs in
+ * proportion to their cost (two blocks : one = 9 : 5); member `slot` of a unit's `group` CTAs takes
+ * the tile_n-column tiles slot + k * group for k < rounds, then its piece
+ * [tail_col0, tail_col0 + tail_cols) of what the whole rounds leave over (cut evenly in 16-column
+ * units; tail_cols may be 0).
+ *   out  host, int32 [10]: {active, two_blocks, first_row_block, slot, group, rounds, tail_col0,
+ *                           tail_cols, thin16, tile_n}
  * Errors: EAD_EINVALID_ARG (also: more row blocks than CTAs).
  */
 int ead_plan_units(int32_t cta, int32_t G, int32_t n_rows, int32_t V, int32_t two_blocks, int32_t *out);

@@ -475,8 +475,8 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
         std::min<size_t>(kMaxStages, (smem_max - kSmemCtrlBytes - 1024 - 1024 - extra) / stage_bytes));
     x->smem_bytes = kSmemCtrlBytes + 1024 + x->stages * stage_bytes + extra;
     if (!x->small_cols) {                          // the kernel cuts the whole ring into 48 or 64 KiB stages per head
-        x->ring_bytes = (smem_max - kSmemCtrlBytes - 2048) & ~static_cast<size_t>(1023);
-        x->smem_bytes = kSmemCtrlBytes + 1024 + x->ring_bytes;
+        x->ring_bytes = (smem_max - kSmemCtrlBytes - 2048 - kThinMergeBytes) & ~static_cast<size_t>(1023);
+        x->smem_bytes = kSmemCtrlBytes + 1024 + x->ring_bytes + kThinMergeBytes;   // merge buffer of the thin block behind the ring
     }
 
     const int B = cfg->B;
@@ -925,6 +925,8 @@ int ead_plan_units(int32_t cta, int32_t G, int32_t n_rows, int32_t V, int32_t tw
     out[5] = s.rounds;
     out[6] = s.tail_col0;
     out[7] = s.tail_cols;
+    out[8] = s.thin16;
+    out[9] = s.tile_n;
     return EAD_OK;
 }
 

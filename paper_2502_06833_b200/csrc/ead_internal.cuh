@@ -104,18 +104,25 @@ __host__ __device__ inline HeadSplit split_head(int cta, int G, int n, int V)
 }
 
 // How the CTAs of the large-batch kernel (B > 128) divide one head.  With n rows there are
-// R = ceil(n / 128) row blocks.  On a head with `two_blocks` set they are taken two at a time:
-// R / 2 units of two blocks and, if R is odd, one unit of the last block alone; otherwise every
-// block is a unit of its own.  Units get CTAs in proportion to their cost (9 : 5 for two blocks :
-// one) and a unit's g CTAs take the head's 256-column tiles round-robin (member `slot` takes
-// tiles slot, slot + g, ...), so that all units sweep the vocabulary at the same pace and a
-// weight tile fetched for one unit is an L2 hit for the others.
+// R = ceil(n / 128) row blocks.  On a head with `two_blocks` set they are taken two at a time
+// (units of two blocks); an odd last block is a unit of its own, or, on a head of three blocks
+// whose last has at most 64 rows, rides along with the two-block unit as a THIN block: its logits are computed with the
+// operands swapped (vocabulary on the MMA's M side, the thin block's rows on N), which takes
+// thin16 = rows rounded up to 16 accumulator columns per 128 vocabulary rows instead of a third
+// 256-column accumulator; the unit's tiles are then tile_n = 256 - thin16 columns wide, so that
+// everything fits the 512 columns of tensor memory.  Without `two_blocks` every block is a unit
+// of its own.  Units get CTAs in proportion to their cost and a unit's g CTAs take the head's
+// tiles round-robin (member `slot` takes tiles slot, slot + g, ...).  Units of the same kind sweep
+// the vocabulary at the same pace, so a weight tile fetched for one is an L2 hit for the others;
+// units of different kinds do not, and a head with two kinds reads its weights twice.
 struct UnitSplit {
     int active;      // this CTA serves a unit of the head
     int dual;        // 1: row blocks rb and rb + 1; 0: row block rb alone
+    int thin16;      // > 0: row block rb + 2 rides along as a thin block of at most thin16 rows
+    int tile_n;      // width of a full tile: 256, or 256 - thin16
     int rb;
     int slot, g;     // member index within the unit's group of g CTAs (also the partial slot)
-    int rounds;      // whole rounds of 256-column tiles: member `slot` takes tile slot + k * g in round k
+    int rounds;      // whole rounds of tile_n-column tiles: member `slot` takes tile slot + k * g in round k
     int tail_col0, tail_cols;   // what is left after the whole rounds is cut evenly (in 16-column
                                 // units) among the g members: this member's piece (tail_cols may be 0)
     int n_tiles;     // pieces this member multiplies: rounds + (tail_cols > 0)
@@ -125,77 +132,107 @@ struct UnitSplit {
 __host__ __device__ inline void unit_piece(const UnitSplit &s, int k, int vpad, int &col0, int &ncols)
 {
     if (k < s.rounds) {
-        col0 = (s.slot + k * s.g) * kTileN;
-        ncols = vpad - col0 < kTileN ? vpad - col0 : kTileN;
+        col0 = (s.slot + k * s.g) * s.tile_n;
+        ncols = vpad - col0 < s.tile_n ? vpad - col0 : s.tile_n;
     } else {
         col0 = s.tail_col0;
         ncols = s.tail_cols;
     }
 }
 
-// Units of a head with n rows (R row blocks): D of two blocks, S of one; CTAs per unit gd and gs,
-// in proportion to what a pipeline stage of the unit costs: measured 1386 cycles for two blocks
-// against 763 for one (18 : 10); a single block of at most 64 rows (an M = 64 tile with half the
-// hidden rows) a little less (9).
-__host__ __device__ inline void unit_groups(int G, int n, int two_blocks, int &D, int &S, int &gd, int &gs)
+// Units of a head with n rows (R row blocks): D of two blocks, then T (0 or 1, and only if D = 0)
+// of two blocks and a thin one, then S of one block; CTAs per unit gd, gt and gs, in proportion to what the unit
+// costs per 256 vocabulary columns and 64 hidden elements: measured 1386 cycles for two blocks
+// against 763 for one (18 : 10), a single block of at most 64 rows (an M = 64 tile with half the
+// hidden rows) a little less (9).  A unit with a thin block is the only unit of its head.
+struct UnitPlan {
+    int D, T, S;
+    int gd, gt, gs;
+    int thin16;
+};
+
+__host__ __device__ inline UnitPlan unit_plan(int G, int n, int two_blocks)
 {
+    UnitPlan u;
+    u.D = u.T = u.S = u.gd = u.gt = u.gs = u.thin16 = 0;
     const int R = (n + kTileM - 1) / kTileM;
-    // Units of different kinds walk the vocabulary at different rates and cannot share a weight
-    // tile in L2, so a head with both kinds reads its weights twice (measured: 3.2 GB per launch
-    // against 2.06 GB).  With three row blocks that makes the head HBM-bound, and three single
-    // units, which share every tile, are faster (917 against 961 us per step at 25 % large rows).
-    D = (two_blocks && R != 3) ? R / 2 : 0;
-    S = R - 2 * D;
-    gd = gs = 0;
-    if (R <= 0) return;
-    const int w_single = (n - (R - 1) * kTileM) <= kTileM / 2 ? 9 : 10;
-    if (D > 0) {
-        gd = (18 * G) / (18 * D + w_single * S);
-        if (gd < 1) gd = 1;
+    if (R <= 0) return u;
+    const int last = n - (R - 1) * kTileM;                   // rows of the last block
+    if (two_blocks && R == 3 && last <= kTileM / 2) {
+        // (with five blocks and more, one two-block unit less and a thin block instead of the
+        // single one measured slower: 1076 against 1055 us per step at 50 % large rows)
+        u.T = 1;
+        u.thin16 = (last + kUnit - 1) / kUnit * kUnit;
+    } else {
+        // Units of different kinds walk the vocabulary at different rates and cannot share a weight
+        // tile in L2, so a head with both kinds reads its weights twice (measured: 3.2 GB per launch
+        // against 2.06 GB).  With three row blocks that makes the head HBM-bound, and three single
+        // units, which share every tile, are faster (917 against 961 us per step at 25 % large rows).
+        u.D = (two_blocks && R != 3) ? R / 2 : 0;
+        u.S = R - 2 * u.D;
     }
-    if (S > 0) {
-        gs = (G - gd * D) / S;
-        if (gs < 1) {                              // fewer CTAs than units are rejected on the host
-            gs = 1;
-            if (D > 0) gd = (G - S) / D > 0 ? (G - S) / D : 1;
+    if (u.T > 0) {
+        u.gt = G;
+        return u;
+    }
+    const int w_single = last <= kTileM / 2 ? 9 : 10;
+    if (u.D > 0) {
+        u.gd = 18 * G / (18 * u.D + w_single * u.S);
+        if (u.gd < 1) u.gd = 1;
+    }
+    const int left = G - u.gd * u.D;                           // CTAs for the single-block units
+    if (u.S > 0) {
+        u.gs = left / u.S;
+        if (u.gs < 1) {                                        // fewer CTAs than units are rejected on the host
+            u.gs = 1;
+            if (u.D > 0) u.gd = (G - u.S) / u.D > 0 ? (G - u.S) / u.D : 1;
         }
     }
+    return u;
 }
 
 __host__ __device__ inline UnitSplit split_units(int cta, int G, int n, int V, int two_blocks)
 {
     UnitSplit s;
-    s.active = 0; s.dual = 0; s.rb = 0; s.slot = 0; s.g = 0;
+    s.active = 0; s.dual = 0; s.thin16 = 0; s.tile_n = kTileN; s.rb = 0; s.slot = 0; s.g = 0;
     s.rounds = 0; s.tail_col0 = 0; s.tail_cols = 0; s.n_tiles = 0;
     if (n <= 0) return s;
-    int D, S, gd, gs;
-    unit_groups(G, n, two_blocks, D, S, gd, gs);
-    if (cta < gd * D) {                            // units interleaved: neighbours in the grid share a slot
+    const UnitPlan u = unit_plan(G, n, two_blocks);
+    const int after_d = u.gd * u.D;
+    if (cta < after_d) {                           // units interleaved: neighbours in the grid share a slot
         s.active = 1;
         s.dual = 1;
-        s.rb = 2 * (cta % D);
-        s.slot = cta / D;
-        s.g = gd;
-    } else if (S > 0 && (cta - gd * D) / S < gs) {
-        const int local = cta - gd * D;
+        s.rb = 2 * (cta % u.D);
+        s.slot = cta / u.D;
+        s.g = u.gd;
+    } else if (u.T > 0 && cta - after_d < u.gt) {
         s.active = 1;
-        s.rb = 2 * D + local % S;
-        s.slot = local / S;
-        s.g = gs;
+        s.dual = 1;
+        s.thin16 = u.thin16;
+        s.tile_n = kTileN - u.thin16;
+        s.rb = 2 * u.D;
+        s.slot = cta - after_d;
+        s.g = u.gt;
+    } else if (u.S > 0 && (cta - after_d) / u.S < u.gs) {
+        const int local = cta - after_d;
+        s.active = 1;
+        s.rb = 2 * u.D + local % u.S;
+        s.slot = local / u.S;
+        s.g = u.gs;
     }
     if (!s.active) return s;
     // Whole rounds of full tiles, then the rest of the vocabulary in g even pieces, so that the
     // members of a unit finish together (with whole tiles only, a unit of 74 CTAs on 594 tiles
     // would wait a ninth round out for two of its members).
     const int vpad = (V + kUnit - 1) / kUnit * kUnit;
-    const int tiles = (V + kTileN - 1) / kTileN;
+    const int tiles = (V + s.tile_n - 1) / s.tile_n;
     s.rounds = tiles / s.g;
-    if (s.rounds * s.g * kTileN > vpad) s.rounds -= 1;       // the last whole round would hold the ragged last tile: deal that round out evenly instead
-    const int rest0 = s.rounds * s.g * kTileN;
-    const int rest = vpad - rest0;                            // < g * 256, a multiple of 16
+    if (s.rounds * s.g * s.tile_n > vpad) s.rounds -= 1;     // the last whole round would hold the ragged last tile: deal that round out evenly instead
+    const int rest0 = s.rounds * s.g * s.tile_n;
+    const int rest = vpad - rest0;                            // < g * tile_n, a multiple of 16
     if (rest > 0) {
         const int units16 = rest / kUnit;
-        const int per = (units16 + s.g - 1) / s.g * kUnit;    // columns per member, a multiple of 16, <= 256
+        const int per = (units16 + s.g - 1) / s.g * kUnit;    // columns per member, a multiple of 16, <= tile_n
         const int c0 = rest0 + s.slot * per;
         if (c0 < vpad) {
             s.tail_col0 = c0;
@@ -209,9 +246,9 @@ __host__ __device__ inline UnitSplit split_units(int cta, int G, int n, int V, i
 // Partial slots that the merge has to fold for compacted row `row` of a head with n rows.
 __host__ __device__ inline int unit_slots_of_row(int G, int n, int row, int two_blocks)
 {
-    int D, S, gd, gs;
-    unit_groups(G, n, two_blocks, D, S, gd, gs);
-    return (row / kTileM) < 2 * D ? gd : gs;
+    const UnitPlan u = unit_plan(G, n, two_blocks);
+    const int rb = row / kTileM;
+    return rb < 2 * u.D ? u.gd : u.T ? u.gt : u.gs;
 }
 
 #ifdef __CUDACC__

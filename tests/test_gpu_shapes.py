@@ -237,6 +237,30 @@ def test_last_row_block_at_the_half_tile_boundary(B, Hl):
     assert np.array_equal(out["tok"][-1], again["tok"][-1])
 
 
+@pytest.mark.parametrize("B,V,temp", [(266, 36000, 0.0), (300, 36000, 0.9), (257, 1900, 0.0), (530, 21000, 0.0),
+                                      (575, 21000, 1.3), (321, 3000, 0.0)])
+def test_short_odd_row_block_rides_along_as_a_thin_block(B, V, temp):
+    """Every row on the large head (hidden size 3072: two-block units).  266 / 300 / 257 rows: two
+    blocks and a third of 10 / 44 / 1 rows, which the kernel multiplies with the operands swapped
+    on tiles of 240 / 208 / 240 columns (whole rounds of tiles at the larger vocabularies, pieces
+    only at 1900); 530 and 575 rows: five blocks, the last one a unit of its own beside two
+    two-block units (575 sampled); 321: a 65-row third block is too long to ride along."""
+    cfg = _cfg(B=B, V=V, H_small=64, H_large=3072, T=2, tau=-1.0, start_model=1, d_min=1)
+    wl = synth.Workload(cfg)
+    seed = 0xABCDEF12345
+    ora = O.run(wl.W_small, wl.W_large, wl.h_small, wl.h_large, w=cfg.w, d_min=cfg.d_min,
+                tau=float(np.float32(cfg.tau)), start_model=1, temperature=temp, seed=seed)
+    with GpuGate(cfg, wl.W_small, wl.W_large, temperature=temp, seed=seed) as g:
+        out = g.run(wl.h_small, wl.h_large, "run")
+        G = g.E.ead_launch_info(g.ctx)["ctas"]
+        plan = g.E.ead_plan_units(G - 1, G, B, V, True)
+    log = compare(out, ora, cfg.tau)
+    assert log["cells"] == B * cfg.T and ora["used"].all()
+    assert len(log["token_near_ties"]) <= 2
+    last = B - (B - 1) // 128 * 128
+    assert (plan["thin16"] > 0) == (last <= 64 and (B + 127) // 128 == 3)
+
+
 def test_a_step_with_every_sequence_ended_computes_nothing_and_keeps_the_state():
     cfg = _cfg(B=150, V=900, T=6, tau=_mid_tau(900))
     wl = synth.Workload(cfg)

@@ -95,14 +95,17 @@ def test_work_split_covers_every_column_once_per_row_block(E, G, n, V):
 
 @pytest.mark.parametrize("G,n,V", [(148, 129, 152064), (148, 256, 152064), (148, 1024, 152064), (148, 266, 152064),
                                    (148, 440, 152064), (148, 4096, 1000), (148, 300, 37), (132, 700, 5000),
-                                   (148, 128, 3000), (20, 1000, 257)])
+                                   (148, 128, 3000), (20, 1000, 257), (148, 532, 152064), (148, 320, 152064),
+                                   (148, 321, 152064), (148, 385, 3000), (148, 257, 100)])
 @pytest.mark.parametrize("two", [True, False])
 def test_unit_split_covers_every_column_once_per_row_block(E, G, n, V, two):
-    """Units of two row blocks (plus one single-block unit for an odd head) or of one block each
-    (always so for a head of three row blocks): every (row block, column) is served by exactly one CTA; a unit's members share its whole
-    rounds of 256-column tiles round-robin and cut the rest evenly, so they finish within 16
-    columns of one another; CTAs are dealt out 9 : 5 between the two kinds of unit."""
+    """Units of two row blocks or of one block each; on a head of three blocks a last block of at
+    most 64 rows rides along with the two-block unit as a thin third block on narrower tiles, and
+    with a fuller last block the head is served one block per unit.  Every (row block, column) is served
+    by exactly one CTA; a unit's members share its whole rounds of tiles round-robin and cut the
+    rest evenly, so they finish within one tile of one another; CTAs are dealt out by unit cost."""
     R = (n + 127) // 128
+    last = n - (R - 1) * 128
     vpad = (V + 15) // 16 * 16
     cover = np.zeros((R, vpad), dtype=np.int32)
     groups, work = {}, {}
@@ -112,34 +115,45 @@ def test_unit_split_covers_every_column_once_per_row_block(E, G, n, V, two):
             continue
         assert 0 <= s["slot"] < s["group"]
         blocks = [s["row_block"], s["row_block"] + 1] if s["two_blocks"] else [s["row_block"]]
+        if s["thin16"]:
+            assert s["two_blocks"] and last <= s["thin16"] <= 64 and s["thin16"] - last < 16
+            blocks.append(s["row_block"] + 2)
+        tn = s["tile_n"]
+        assert tn == 256 - s["thin16"]
         assert s["row_block"] % 2 == 0 or not s["two_blocks"]
-        cols = 0
         for rb in blocks:
             assert 0 <= rb < R
             for k in range(s["rounds"]):
-                c0 = (s["slot"] + k * s["group"]) * 256
+                c0 = (s["slot"] + k * s["group"]) * tn
                 assert c0 < vpad
-                cover[rb, c0:min(vpad, c0 + 256)] += 1
+                cover[rb, c0:min(vpad, c0 + tn)] += 1
             if s["tail_cols"]:
-                assert s["tail_cols"] % 16 == 0 and s["tail_col0"] % 16 == 0 and 0 < s["tail_cols"] <= 256
+                assert s["tail_cols"] % 16 == 0 and s["tail_col0"] % 16 == 0 and 0 < s["tail_cols"] <= tn
                 cover[rb, s["tail_col0"]:s["tail_col0"] + s["tail_cols"]] += 1
-        cols = min(vpad, s["rounds"] * 256) if s["rounds"] else 0
-        key = (s["row_block"], s["two_blocks"])
+        key = (s["row_block"], s["two_blocks"], s["thin16"])
         groups.setdefault(key, set()).add(s["slot"])
-        work.setdefault(key, []).append(s["rounds"] * 256 + s["tail_cols"])
+        work.setdefault(key, []).append(s["rounds"] * tn + s["tail_cols"])
     assert (cover == 1).all(), "a column of a row block is missed or served twice"
     for key, w in work.items():
         if V >= 256 * len(w):                                    # enough columns for whole rounds
             assert max(w) - min([x for x in w if x] or [0]) <= 256, (key, sorted(set(w)))
     kinds = {k: len(v) for k, v in groups.items()}
-    duals = [v for (rb, two_), v in kinds.items() if two_]
-    singles = [v for (rb, two_), v in kinds.items() if not two_]
-    n_dual = R // 2 if two and R != 3 else 0
-    assert len(duals) == n_dual and len(singles) == R - 2 * n_dual
+    duals = [v for (rb, two_, thin), v in kinds.items() if two_ and not thin]
+    thins = [v for (rb, two_, thin), v in kinds.items() if thin]
+    singles = [v for (rb, two_, thin), v in kinds.items() if not two_]
+    if two and R == 3 and last <= 64:
+        want = (0, 1, 0)
+    elif two and R != 3:
+        want = (R // 2, 0, R % 2)
+    else:
+        want = (0, 0, R)
+    assert (len(duals), len(thins), len(singles)) == want
     assert len(set(duals)) <= 1 and len(set(singles)) <= 1       # units of a kind are alike
     if duals and singles and G >= 40:
         assert 0.4 <= singles[0] / duals[0] <= 0.75             # about 5 : 9
-    assert sum(duals) + sum(singles) <= G
+    if thins:
+        assert thins == [G] and not duals and not singles       # a unit with a thin block has the head to itself
+    assert sum(duals) + sum(thins) + sum(singles) <= G
     with pytest.raises(E.EadError):
         E.ead_plan_units(0, 4, 1000, 257, two)                   # eight row blocks, four CTAs
 
