@@ -262,10 +262,10 @@ def ead_plan_split(cta, G, n_rows, V) -> dict:
 
 
 def ead_plan_units(cta, G, n_rows, V, two_blocks=True) -> dict:
-    a = (C.c_int32 * 10)()
+    a = (C.c_int32 * 13)()
     _check(lib().ead_plan_units(int(cta), int(G), int(n_rows), int(V), int(bool(two_blocks)), a), "ead_plan_units")
     return dict(active=a[0], two_blocks=a[1], row_block=a[2], slot=a[3], group=a[4], rounds=a[5],
-                tail_col0=a[6], tail_cols=a[7], thin16=a[8], tile_n=a[9])
+                tail_col0=a[6], tail_cols=a[7], thin16=a[8], tile_n=a[9], n_hi=a[10], w_hi=a[11], w_lo=a[12])
 
 
 def ead_shard_range(V, n_shards, shard) -> tuple:

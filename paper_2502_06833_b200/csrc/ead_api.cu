@@ -97,7 +97,7 @@ struct ead_ctx {
     uint16_t *hc[2] = {nullptr, nullptr};
     ShardLink *link = nullptr;             // vocabulary-sharded contexts: where the records go (device)
     bool connected = false;                // ead_shard_connect has filled `link`
-    CUtensorMap tmA[2], tmH[2], tmW[2], tmT[2], tmP[2];   // hidden rows (boxes of a_rows and of 64 rows); W boxes of 256|128, 16 and 32 rows
+    CUtensorMap tmA[2], tmH[2], tmW[2], tmT[2], tmP[2], tmQ[2];   // hidden rows (boxes of a_rows and of 64 rows); W boxes of 256|128, 16, 32 and 64 rows
     cudaGraphExec_t g_one = nullptr, g_chunk = nullptr;
     int64_t launches = 0;
     // staging of ead_run_host (allocated on first use)
@@ -236,9 +236,9 @@ int enqueue_step(ead_ctx *x, cudaStream_t s, cudaEvent_t *ev = nullptr, int shar
             lp.two_blocks = x->two_blocks;
             lp.ring_bytes = static_cast<int32_t>(x->ring_bytes);
             e = lp.sampling ? launch(ead_lmhead_dual_kernel<true>, lgrid, lblock, x->smem_bytes, s, pdl, x->tmA[0],
-                                     x->tmA[1], x->tmW[0], x->tmW[1], x->tmT[0], x->tmT[1], x->tmH[0], x->tmH[1], lp)
+                                     x->tmA[1], x->tmW[0], x->tmW[1], x->tmT[0], x->tmT[1], x->tmH[0], x->tmH[1], x->tmQ[0], x->tmQ[1], lp)
                             : launch(ead_lmhead_dual_kernel<false>, lgrid, lblock, x->smem_bytes, s, pdl, x->tmA[0],
-                                     x->tmA[1], x->tmW[0], x->tmW[1], x->tmT[0], x->tmT[1], x->tmH[0], x->tmH[1], lp);
+                                     x->tmA[1], x->tmW[0], x->tmW[1], x->tmT[0], x->tmT[1], x->tmH[0], x->tmH[1], x->tmQ[0], x->tmQ[1], lp);
             break;
         case 1: EAD_LAUNCH_SMALL(1); break;
         case 2: EAD_LAUNCH_SMALL(2); break;
@@ -527,7 +527,9 @@ int ead_create(const ead_config *cfg, const void *W_small, const void *W_large, 
             !encode_bf16_2d(&x->tmH[m], x->hc[m], Bpad, Hm[m], std::min(x->a_rows, kTileM / 2)) ||
             !encode_bf16_2d(&x->tmW[m], x->W[m], Vm[m], Hm[m], wbox) ||
             !encode_bf16_2d(&x->tmT[m], x->W[m], Vm[m], Hm[m], kUnit) ||
-            !encode_bf16_2d(&x->tmP[m], x->W[m], Vm[m], Hm[m], kSmallSegRows))
+            !encode_bf16_2d(&x->tmP[m], x->W[m], Vm[m], Hm[m], kSmallSegRows) ||
+            !encode_bf16_2d(&x->tmQ[m], x->W[m], Vm[m], Hm[m],
+                            static_cast<uint32_t>(std::min(64, (Vm[m] + kUnit - 1) / kUnit * kUnit))))
             return fail(EAD_ECUDA);
     }
     // the attribute belongs to the kernel on this device, not to the context: ask for the
@@ -927,6 +929,9 @@ int ead_plan_units(int32_t cta, int32_t G, int32_t n_rows, int32_t V, int32_t tw
     out[7] = s.tail_cols;
     out[8] = s.thin16;
     out[9] = s.tile_n;
+    out[10] = s.n_hi;
+    out[11] = s.w_hi;
+    out[12] = s.w_lo;
     return EAD_OK;
 }
 

@@ -122,18 +122,31 @@ struct UnitSplit {
     int tile_n;      // width of a full tile: 256, or 256 - thin16
     int rb;
     int slot, g;     // member index within the unit's group of g CTAs (also the partial slot)
-    int rounds;      // whole rounds of tile_n-column tiles: member `slot` takes tile slot + k * g in round k
+    int rounds;      // whole rounds of tiles: member `slot` takes tile slot + k * g in round k.  The first
+    int n_hi;        // n_hi rounds have tiles of w_hi columns, the others of w_lo (both multiples of 16,
+    int w_hi, w_lo;  // at most tile_n)
     int tail_col0, tail_cols;   // what is left after the whole rounds is cut evenly (in 16-column
                                 // units) among the g members: this member's piece (tail_cols may be 0)
     int n_tiles;     // pieces this member multiplies: rounds + (tail_cols > 0)
 };
 
+// On a head of three row blocks and more, a member's share in few pieces (at most this many whole
+// rounds of full tiles) is cut into pieces of nearly equal width instead of full tiles and a
+// narrow last one that only some members have (measured: step at 25 % large rows 843 -> 824 us,
+// at 50 % 1079 -> 1048 us).  A head of one or two row blocks streams its weights from HBM at the
+// rate its loads in flight allow, and narrower tiles mean fewer bytes in flight: there the
+// full tiles stay (B = 256 step with them 393 us, with even pieces 420 us).
+constexpr int kEvenRoundsMax = 8;
+constexpr int kEvenRoundsMinBlocks = 3;
+
 // Column range [col0, col0 + ncols) of piece k (0 <= k < n_tiles) of a member; vpad = V rounded up to 16.
 __host__ __device__ inline void unit_piece(const UnitSplit &s, int k, int vpad, int &col0, int &ncols)
 {
     if (k < s.rounds) {
-        col0 = (s.slot + k * s.g) * s.tile_n;
-        ncols = vpad - col0 < s.tile_n ? vpad - col0 : s.tile_n;
+        const int hi = k < s.n_hi ? k : s.n_hi;              // rounds of the wider kind before this one
+        const int w = k < s.n_hi ? s.w_hi : s.w_lo;
+        col0 = s.g * (hi * s.w_hi + (k - hi) * s.w_lo) + s.slot * w;
+        ncols = vpad - col0 < w ? vpad - col0 : w;
     } else {
         col0 = s.tail_col0;
         ncols = s.tail_cols;
@@ -195,7 +208,7 @@ __host__ __device__ inline UnitSplit split_units(int cta, int G, int n, int V, i
 {
     UnitSplit s;
     s.active = 0; s.dual = 0; s.thin16 = 0; s.tile_n = kTileN; s.rb = 0; s.slot = 0; s.g = 0;
-    s.rounds = 0; s.tail_col0 = 0; s.tail_cols = 0; s.n_tiles = 0;
+    s.rounds = 0; s.n_hi = 0; s.w_hi = s.w_lo = kTileN; s.tail_col0 = 0; s.tail_cols = 0; s.n_tiles = 0;
     if (n <= 0) return s;
     const UnitPlan u = unit_plan(G, n, two_blocks);
     const int after_d = u.gd * u.D;
@@ -225,11 +238,26 @@ __host__ __device__ inline UnitSplit split_units(int cta, int G, int n, int V, i
     // members of a unit finish together (with whole tiles only, a unit of 74 CTAs on 594 tiles
     // would wait a ninth round out for two of its members).
     const int vpad = (V + kUnit - 1) / kUnit * kUnit;
+    const int U = vpad / kUnit;                               // 16-column units of the head
+    const int tile_u = s.tile_n / kUnit;
     const int tiles = (V + s.tile_n - 1) / s.tile_n;
     s.rounds = tiles / s.g;
+    s.w_hi = s.w_lo = s.tile_n;
     if (s.rounds * s.g * s.tile_n > vpad) s.rounds -= 1;     // the last whole round would hold the ragged last tile: deal that round out evenly instead
-    const int rest0 = s.rounds * s.g * s.tile_n;
-    const int rest = vpad - rest0;                            // < g * tile_n, a multiple of 16
+    s.n_hi = s.rounds;
+    if (n > (kEvenRoundsMinBlocks - 1) * kTileM && s.rounds >= 1 && s.rounds <= kEvenRoundsMax &&
+        U > s.rounds * s.g * tile_u) {
+        // few pieces: n_p pieces of nearly equal width, the last one again the even rest
+        const int u_tot = (U + s.g - 1) / s.g;                // units of the member with the most
+        const int n_p = (u_tot + tile_u - 1) / tile_u;
+        const int base = u_tot / n_p, extra = u_tot % n_p;    // `extra` pieces of base + 1 units, the others of base
+        s.rounds = n_p - 1;
+        s.n_hi = extra < s.rounds ? extra : s.rounds;
+        s.w_hi = (base + 1) * kUnit;
+        s.w_lo = base * kUnit;
+    }
+    const int rest0 = s.g * (s.n_hi * s.w_hi + (s.rounds - s.n_hi) * s.w_lo);
+    const int rest = vpad - rest0;                            // a multiple of 16
     if (rest > 0) {
         const int units16 = rest / kUnit;
         const int per = (units16 + s.g - 1) / s.g * kUnit;    // columns per member, a multiple of 16, <= tile_n

@@ -72,11 +72,13 @@ struct HeadRing {
 };
 
 #ifdef __CUDACC__
-__device__ __forceinline__ HeadRing head_ring(const LmheadParams &p, const UnitSplit &sp)
+__device__ __forceinline__ HeadRing head_ring(const LmheadParams &p, const UnitSplit &sp, bool half_single)
 {
     HeadRing r;
-    r.stage_bytes = sp.thin16 ? kThinStageBytes : sp.dual ? kDualStageBytes : kSingleStageBytes;
-    r.w_off = sp.thin16 ? 2 * kDualABytes + kThinABytes : sp.dual ? 2 * kDualABytes : kDualABytes;
+    // (a single block of at most 64 rows brings in 8 KiB of hidden rows per stage: 40 KiB stages, five of them)
+    const uint32_t single_a = half_single ? kDualABytes / 2 : kDualABytes;
+    r.stage_bytes = sp.thin16 ? kThinStageBytes : sp.dual ? kDualStageBytes : single_a + kWTileBytes;
+    r.w_off = sp.thin16 ? 2 * kDualABytes + kThinABytes : sp.dual ? 2 * kDualABytes : single_a;
     r.stages = min(kMaxStages, static_cast<int>(static_cast<uint32_t>(p.ring_bytes) / r.stage_bytes));
     return r;
 }
@@ -175,13 +177,14 @@ __device__ __forceinline__ BlockView block_view(const LmheadParams &p, int n, in
 }
 
 // tmA*: compacted hidden rows, boxes of 128 x 64; tmH*: the same, boxes of 64 x 64; tmW*: W, boxes
-// of 256 x 64; tmT*: W, boxes of 16 x 64 (ragged last tile).
+// of 256 x 64; tmQ*, tmT*: W, boxes of 64 x 64 and 16 x 64 (pieces narrower than a tile).
 template <bool SAMPLE>
 __global__ void __launch_bounds__(kLmheadThreads, 1)
 ead_lmhead_dual_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
                        const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
                        const __grid_constant__ CUtensorMap tmT0, const __grid_constant__ CUtensorMap tmT1,
                        const __grid_constant__ CUtensorMap tmH0, const __grid_constant__ CUtensorMap tmH1,
+                       const __grid_constant__ CUtensorMap tmQ0, const __grid_constant__ CUtensorMap tmQ1,
                        const LmheadParams p)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -213,6 +216,7 @@ ead_lmhead_dual_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
         tma_prefetch_desc(&tmW0); tma_prefetch_desc(&tmW1);
         tma_prefetch_desc(&tmT0); tma_prefetch_desc(&tmT1);
         tma_prefetch_desc(&tmH0); tma_prefetch_desc(&tmH1);
+        tma_prefetch_desc(&tmQ0); tma_prefetch_desc(&tmQ1);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&ctrl->tmem_base), 2 * kTileN);
@@ -239,7 +243,9 @@ ead_lmhead_dual_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
             for (int m = 0; m < 2 && ok; ++m) {
                 const UnitSplit sp = split_units(cta, G, n_rows[m], p.V[m], (p.two_blocks >> m) & 1);
                 if (!sp.active) continue;
-                const HeadRing ring = head_ring(p, sp);
+                const BlockView ba = block_view(p, n_rows[m], sp.rb, true);
+                const BlockView bb = block_view(p, n_rows[m], sp.rb + 1, sp.dual != 0);
+                const HeadRing ring = head_ring(p, sp, !sp.dual && ba.half);
                 // The ring may be cut differently for this head: every stage filled so far must have
                 // been consumed first (the wait a refill of the slot would do; a slot never filled
                 // passes at once).
@@ -249,8 +255,7 @@ ead_lmhead_dual_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                 uint32_t s = 0;
                 const CUtensorMap *tW = m ? &tmW1 : &tmW0;
                 const CUtensorMap *tT = m ? &tmT1 : &tmT0;
-                const BlockView ba = block_view(p, n_rows[m], sp.rb, true);
-                const BlockView bb = block_view(p, n_rows[m], sp.rb + 1, sp.dual != 0);
+                const CUtensorMap *tQ = m ? &tmQ1 : &tmQ0;
                 const CUtensorMap *tAa = ba.half ? (m ? &tmH1 : &tmH0) : (m ? &tmA1 : &tmA0);
                 const CUtensorMap *tAb = bb.half ? (m ? &tmH1 : &tmH0) : (m ? &tmA1 : &tmA0);
                 const CUtensorMap *tAc = m ? &tmH1 : &tmH0;
@@ -277,8 +282,11 @@ ead_lmhead_dual_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                         const uint32_t sw = sa + ring.w_off;
                         if (full) {
                             tma_load_2d(sw, tW, kb * kBlockK, col0, bar, pol_w);
-                        } else {
-                            for (int j = 0; j < ncols; j += kUnit)
+                        } else {                     // exactly the piece's rows: boxes of 64, then of 16
+                            int j = 0;
+                            for (; ncols - j >= 64; j += 64)
+                                tma_load_2d(sw + j * (kBlockK * 2), tQ, kb * kBlockK, col0 + j, bar, pol_w);
+                            for (; j < ncols; j += kUnit)
                                 tma_load_2d(sw + j * (kBlockK * 2), tT, kb * kBlockK, col0 + j, bar, pol_w);
                         }
                         par ^= 1u << s;
@@ -301,10 +309,10 @@ ead_lmhead_dual_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
             for (int m = 0; m < 2 && ok; ++m) {
                 const UnitSplit sp = split_units(cta, G, n_rows[m], p.V[m], (p.two_blocks >> m) & 1);
                 if (!sp.active) continue;
-                const HeadRing ring = head_ring(p, sp);
-                uint32_t s = 0;
                 const BlockView ba = block_view(p, n_rows[m], sp.rb, true);
                 const BlockView bb = block_view(p, n_rows[m], sp.rb + 1, sp.dual != 0);
+                const HeadRing ring = head_ring(p, sp, !sp.dual && ba.half);
+                uint32_t s = 0;
                 const int kblocks = (p.H[m] + kBlockK - 1) / kBlockK;
                 const int vpad = (p.V[m] + kUnit - 1) / kUnit * kUnit;
                 for (int t = 0; t < sp.n_tiles && ok; ++t) {

@@ -123,16 +123,25 @@ def test_unit_split_covers_every_column_once_per_row_block(E, G, n, V, two):
         assert s["row_block"] % 2 == 0 or not s["two_blocks"]
         for rb in blocks:
             assert 0 <= rb < R
+            mine = 0
             for k in range(s["rounds"]):
-                c0 = (s["slot"] + k * s["group"]) * tn
+                hi = min(k, s["n_hi"])
+                wk = s["w_hi"] if k < s["n_hi"] else s["w_lo"]
+                assert 16 <= wk <= tn and wk % 16 == 0
+                c0 = s["group"] * (hi * s["w_hi"] + (k - hi) * s["w_lo"]) + s["slot"] * wk
                 assert c0 < vpad
-                cover[rb, c0:min(vpad, c0 + tn)] += 1
+                cover[rb, c0:min(vpad, c0 + wk)] += 1
+                mine += min(vpad, c0 + wk) - c0
             if s["tail_cols"]:
                 assert s["tail_cols"] % 16 == 0 and s["tail_col0"] % 16 == 0 and 0 < s["tail_cols"] <= tn
                 cover[rb, s["tail_col0"]:s["tail_col0"] + s["tail_cols"]] += 1
         key = (s["row_block"], s["two_blocks"], s["thin16"])
         groups.setdefault(key, set()).add(s["slot"])
-        work.setdefault(key, []).append(s["rounds"] * tn + s["tail_cols"])
+        work.setdefault(key, []).append(mine + s["tail_cols"])
+        if s["rounds"] and (s["w_hi"], s["w_lo"]) != (tn, tn):   # a share in few pieces: all of about the same width
+            assert s["rounds"] <= 8 and s["w_hi"] == s["w_lo"] + 16 and R >= 3
+            assert s["tail_cols"] == 0 or s["w_lo"] - 16 <= s["tail_cols"] <= s["w_lo"] or s["slot"] == s["group"] - 1 \
+                or s["tail_col0"] + s["tail_cols"] == vpad
     assert (cover == 1).all(), "a column of a row block is missed or served twice"
     for key, w in work.items():
         if V >= 256 * len(w):                                    # enough columns for whole rounds
