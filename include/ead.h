@@ -312,8 +312,9 @@ int ead_plan_split(int32_t cta, int32_t G, int32_t n_rows, int32_t V, int32_t *o
  * what the whole rounds leave over (cut evenly in 16-column units; tail_cols may be 0).  The
  * tiles of the first n_hi rounds are w_hi columns wide, those of the other rounds w_lo (round k
  * begins where round k - 1 ends: at group * (min(k, n_hi) * w_hi + max(0, k - n_hi) * w_lo)).  With
- * more than eight whole rounds of full tiles, no rest, or a head of at most two row blocks, all
- * are tile_n wide; otherwise a member's share is cut into pieces of nearly equal width.
+ * more than eight whole rounds of full tiles, no rest, or single-block units on a head of at most
+ * two row blocks, all are tile_n wide; otherwise a member's share is cut into pieces of nearly
+ * equal width.
  *   out  host, int32 [13]: {active, two_blocks, first_row_block, slot, group, rounds, tail_col0,
  *                           tail_cols, thin16, tile_n, n_hi, w_hi, w_lo}
  * Errors: EAD_EINVALID_ARG (also: more row blocks than CTAs).

@@ -130,12 +130,14 @@ struct UnitSplit {
     int n_tiles;     // pieces this member multiplies: rounds + (tail_cols > 0)
 };
 
-// On a head of three row blocks and more, a member's share in few pieces (at most this many whole
-// rounds of full tiles) is cut into pieces of nearly equal width instead of full tiles and a
-// narrow last one that only some members have (measured: step at 25 % large rows 843 -> 824 us,
-// at 50 % 1079 -> 1048 us).  A head of one or two row blocks streams its weights from HBM at the
-// rate its loads in flight allow, and narrower tiles mean fewer bytes in flight: there the
-// full tiles stay (B = 256 step with them 393 us, with even pieces 420 us).
+// A member's share in few pieces (at most this many whole rounds of full tiles) is cut into
+// pieces of nearly equal width instead of full tiles and a narrow last one that only some
+// members have: on a head of three row blocks and more (measured: step at 25 % large rows
+// 843 -> 824 us, at 50 % 1079 -> 1048 us, 300 rows on the small head 144 -> 134 us) and in a
+// two-block unit (181 rows on the large head 326 -> 304 us).  Single-block units of a head of one
+// or two blocks stream their weights from HBM at the rate their loads in flight allow, and
+// narrower tiles in several boxes mean fewer bytes in flight: there the full tiles stay (256 rows
+// on the small head 103 us with them, 144 us with even pieces).
 constexpr int kEvenRoundsMax = 8;
 constexpr int kEvenRoundsMinBlocks = 3;
 
@@ -245,7 +247,7 @@ __host__ __device__ inline UnitSplit split_units(int cta, int G, int n, int V, i
     s.w_hi = s.w_lo = s.tile_n;
     if (s.rounds * s.g * s.tile_n > vpad) s.rounds -= 1;     // the last whole round would hold the ragged last tile: deal that round out evenly instead
     s.n_hi = s.rounds;
-    if (n > (kEvenRoundsMinBlocks - 1) * kTileM && s.rounds >= 1 && s.rounds <= kEvenRoundsMax &&
+    if ((n > (kEvenRoundsMinBlocks - 1) * kTileM || s.dual) && s.rounds >= 1 && s.rounds <= kEvenRoundsMax &&
         U > s.rounds * s.g * tile_u) {
         // few pieces: n_p pieces of nearly equal width, the last one again the even rest
         const int u_tot = (U + s.g - 1) / s.g;                // units of the member with the most

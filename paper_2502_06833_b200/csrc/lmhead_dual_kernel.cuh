@@ -72,11 +72,14 @@ struct HeadRing {
 };
 
 #ifdef __CUDACC__
-__device__ __forceinline__ HeadRing head_ring(const LmheadParams &p, const UnitSplit &sp, bool half_single)
+__device__ __forceinline__ HeadRing head_ring(const LmheadParams &p, const UnitSplit &sp, bool half_head)
 {
     HeadRing r;
-    // (a single block of at most 64 rows brings in 8 KiB of hidden rows per stage: 40 KiB stages, five of them)
-    const uint32_t single_a = half_single ? kDualABytes / 2 : kDualABytes;
+    // A head of at most 64 rows brings in 8 KiB of hidden rows per stage: 40 KiB stages, five of
+    // them.  (Not so a short block beside other blocks of its head: units that share their weight
+    // tiles through L2 must move in step, and with rings of different depth they do not; measured
+    // on 181 rows of the small head: 101 us with equal stages, 148 us with 48 and 40 KiB ones.)
+    const uint32_t single_a = half_head ? kDualABytes / 2 : kDualABytes;
     r.stage_bytes = sp.thin16 ? kThinStageBytes : sp.dual ? kDualStageBytes : single_a + kWTileBytes;
     r.w_off = sp.thin16 ? 2 * kDualABytes + kThinABytes : sp.dual ? 2 * kDualABytes : single_a;
     r.stages = min(kMaxStages, static_cast<int>(static_cast<uint32_t>(p.ring_bytes) / r.stage_bytes));
@@ -245,7 +248,7 @@ ead_lmhead_dual_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                 if (!sp.active) continue;
                 const BlockView ba = block_view(p, n_rows[m], sp.rb, true);
                 const BlockView bb = block_view(p, n_rows[m], sp.rb + 1, sp.dual != 0);
-                const HeadRing ring = head_ring(p, sp, !sp.dual && ba.half);
+                const HeadRing ring = head_ring(p, sp, n_rows[m] <= kTileM / 2);
                 // The ring may be cut differently for this head: every stage filled so far must have
                 // been consumed first (the wait a refill of the slot would do; a slot never filled
                 // passes at once).
@@ -311,7 +314,7 @@ ead_lmhead_dual_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                 if (!sp.active) continue;
                 const BlockView ba = block_view(p, n_rows[m], sp.rb, true);
                 const BlockView bb = block_view(p, n_rows[m], sp.rb + 1, sp.dual != 0);
-                const HeadRing ring = head_ring(p, sp, !sp.dual && ba.half);
+                const HeadRing ring = head_ring(p, sp, n_rows[m] <= kTileM / 2);
                 uint32_t s = 0;
                 const int kblocks = (p.H[m] + kBlockK - 1) / kBlockK;
                 const int vpad = (p.V[m] + kUnit - 1) / kUnit * kUnit;

@@ -139,7 +139,7 @@ def test_unit_split_covers_every_column_once_per_row_block(E, G, n, V, two):
         groups.setdefault(key, set()).add(s["slot"])
         work.setdefault(key, []).append(mine + s["tail_cols"])
         if s["rounds"] and (s["w_hi"], s["w_lo"]) != (tn, tn):   # a share in few pieces: all of about the same width
-            assert s["rounds"] <= 8 and s["w_hi"] == s["w_lo"] + 16 and R >= 3
+            assert s["rounds"] <= 8 and s["w_hi"] == s["w_lo"] + 16 and (R >= 3 or s["two_blocks"])
             assert s["tail_cols"] == 0 or s["w_lo"] - 16 <= s["tail_cols"] <= s["w_lo"] or s["slot"] == s["group"] - 1 \
                 or s["tail_col0"] + s["tail_cols"] == vpad
     assert (cover == 1).all(), "a column of a row block is missed or served twice"
