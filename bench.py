@@ -65,13 +65,15 @@ TARGET_TIMED_SECONDS = 0.25          # repeats are added until the timed regions
 # with the same live heads; workloads whose steps differ mix the per-head figures.
 NCU_DRAM_BYTES_PER_LAUNCH = {
     ("llama_b1", "large"): (1.05726e9, "profiles/lmhead_small_kernel_llama_b1_ncu_full.md"),
-    ("llama_b1", "small"): (5.3285e8, "profiles/lmhead_kernels_other_configs_ncu_counters.md"),
+    ("llama_b1", "small"): (5.3285e8, "profiles/lmhead_small_kernel_llama_b1_small_only_ncu_counters.md"),
     ("llama_b64", "both"): (1.5823e9, "profiles/lmhead_small_kernel_llama_b64_ncu_full.md"),
-    ("qwen_b256", "both"): (2.0384e9, "profiles/lmhead_kernel_qwen_b256_ncu_counters.md"),
-    ("qwen_b1024", "small"): (4.7385e8, "profiles/lmhead_kernels_other_configs_ncu_counters.md"),
-    # captured at 25 % and 50 % of the rows on the large head (2.0677 and 2.0622 GB): their mean
-    ("qwen_b1024", "both"): (2.0649e9, "profiles/lmhead_kernels_other_configs_ncu_counters.md"),
-    ("qwen_b1024", "large"): (1.6049e9, "profiles/lmhead_kernel_qwen_b1024_all_large_ncu_full.md"),
+    ("qwen_b256", "both"): (2.0305e9, "profiles/lmhead_dual_kernel_qwen_configs_ncu_counters.md"),
+    ("qwen_b1024", "small"): (4.7428e8, "profiles/lmhead_dual_kernel_qwen_configs_ncu_counters.md"),
+    # with both heads live the traffic depends on how the large head's row blocks fall into units
+    # (one pass over its weights per kind of unit): keyed by configuration, not by family
+    ("qwen_b1024_f25", "both"): (2.0606e9, "profiles/lmhead_dual_kernel_qwen_configs_ncu_counters.md"),
+    ("qwen_b1024_f50", "both"): (2.9448e9, "profiles/lmhead_dual_kernel_qwen_configs_ncu_counters.md"),
+    ("qwen_b1024", "large"): (1.6573e9, "profiles/lmhead_dual_kernel_qwen_configs_ncu_counters.md"),
 }
 
 
@@ -215,7 +217,7 @@ def ncu_traffic(cfg, used: np.ndarray):
         share = float((kinds == code).mean())
         if share == 0.0:
             continue
-        entry = NCU_DRAM_BYTES_PER_LAUNCH.get((family, kind))
+        entry = NCU_DRAM_BYTES_PER_LAUNCH.get((cfg.name, kind)) or NCU_DRAM_BYTES_PER_LAUNCH.get((family, kind))
         if entry is None:
             return None, None
         total += share * entry[0]
@@ -435,7 +437,7 @@ def measure(rt: Runtime, cfg, K: int, W: int, repeats: int | None, temperature: 
     traffic, files = ncu_traffic(cfg, used_np[W:])
     roof["traffic"] = traffic
     roof["traffic_source"] = files
-    roof.update({"kernel": "ead_lmhead_small_kernel" if B <= 128 else "ead_lmhead_kernel",
+    roof.update({"kernel": "ead_lmhead_small_kernel" if B <= 128 else "ead_lmhead_dual_kernel",
                  "kernel_us_per_launch": t_kernel * 1e6,
                  "algorithmic_bytes_per_launch": bytes_s.mean(), "flops_per_launch": flops_s.mean(),
                  "other_kernels_us_per_step": float(np.median(

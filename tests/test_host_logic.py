@@ -212,7 +212,8 @@ def test_bench_ncu_traffic_follows_the_heads_that_were_live():
     used = np.zeros((4, cfg.B), dtype=np.uint8)
     used[:, :300] = 1                                                   # both heads live in every step
     got, files = bench.ncu_traffic(cfg, used)
-    assert got == pytest.approx(tab[("qwen_b1024", "both")][0])
+    assert got == pytest.approx(tab[("qwen_b1024_f25", "both")][0])     # mixed steps: keyed by configuration
+    assert tab[("qwen_b1024_f50", "both")][0] > 1.3 * got               # ... because the unit layout sets the traffic
     used[:] = 1
     assert bench.ncu_traffic(cfg, used)[0] == pytest.approx(tab[("qwen_b1024", "large")][0])
     assert bench.ncu_traffic(configs.TINY, np.zeros((2, 4), dtype=np.uint8)) == (None, None)   # never captured
