@@ -362,7 +362,8 @@ __device__ __forceinline__ Partial warp_merge(Partial acc)
     return acc;
 }
 
-// One warp per compacted row: partials of ead_lmhead_kernel (one slot per CTA of the row's group).
+// One warp per compacted row: partials of the large-batch LM-head kernels (one slot per CTA of the
+// row's group, or per member of the unit that serves the row).
 __global__ void __launch_bounds__(kGateThreads) ead_merge_gate_kernel(const GateParams p)
 {
     const int lane = threadIdx.x & 31;
