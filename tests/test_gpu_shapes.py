@@ -238,13 +238,15 @@ def test_last_row_block_at_the_half_tile_boundary(B, Hl):
 
 
 @pytest.mark.parametrize("B,V,temp", [(266, 36000, 0.0), (300, 36000, 0.9), (257, 1900, 0.0), (530, 21000, 0.0),
-                                      (575, 21000, 1.3), (321, 3000, 0.0)])
+                                      (575, 21000, 1.3), (321, 3000, 0.0), (313, 35991, 0.0), (290, 35991, 1.1)])
 def test_short_odd_row_block_rides_along_as_a_thin_block(B, V, temp):
     """Every row on the large head (hidden size 3072: two-block units).  266 / 300 / 257 rows: two
     blocks and a third of 10 / 44 / 1 rows, which the kernel multiplies with the operands swapped
     on tiles of 240 / 208 / 240 columns (whole rounds of tiles at the larger vocabularies, pieces
     only at 1900); 530 and 575 rows: five blocks, the last one a unit of its own beside two
-    two-block units (575 sampled); 321: a 65-row third block is too long to ride along."""
+    two-block units (575 sampled); 321: a 65-row third block is too long to ride along; 313 and
+    290 rows on a vocabulary that is no multiple of 16: thin blocks of 57 rows (tiles of 192 columns,
+    the second thin accumulator starting at tile row 64) and of 34 rows, sampled."""
     cfg = _cfg(B=B, V=V, H_small=64, H_large=3072, T=2, tau=-1.0, start_model=1, d_min=1)
     wl = synth.Workload(cfg)
     seed = 0xABCDEF12345
