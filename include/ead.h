@@ -144,7 +144,7 @@ int ead_run_host(ead_ctx *ctx, int32_t T, const void *h_small_seq, const void *h
 
 /*
  * DIAGNOSTIC (measurement aid, not part of the gate step's interface; so are
- * ead_kernel_launches, ead_launch_info and ead_plan_split below).
+ * ead_kernel_launches, ead_launch_info, ead_plan_split and ead_plan_units below).
  * The same T steps as ead_run, launched kernel by kernel (no graph replay) with
  * CUDA events around every kernel on cfg.stream, to attribute device time.
  *   kernel_ms  host, float [3]: summed device time in milliseconds of the
@@ -214,7 +214,9 @@ int64_t ead_kernel_launches(const ead_ctx *ctx);
 
 /* DIAGNOSTIC.  Launch geometry chosen at creation, for reporting: fills up to n ints with
  * {CTAs of the LM-head kernel, pipeline stages, rows of the hidden-state TMA
- * box, dynamic shared memory bytes}. */
+ * box, dynamic shared memory bytes}.  For B > 128 the stage count is that of a single-block unit
+ * (48 KiB stages); the kernel cuts the same ring into 64 or 72 KiB stages for units of two blocks
+ * and into 40 KiB ones for a head of at most 64 rows. */
 int ead_launch_info(const ead_ctx *ctx, int32_t *info, int32_t n);
 
 /*
