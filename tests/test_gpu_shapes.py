@@ -263,6 +263,18 @@ def test_short_odd_row_block_rides_along_as_a_thin_block(B, V, temp):
     assert (plan["thin16"] > 0) == (last <= 64 and (B + 127) // 128 == 3)
 
 
+def test_thin_block_on_the_small_head_with_the_large_head_idle():
+    """The same unit on head 0: every row stays on a small head whose hidden size is long enough
+    for two-block units (266 rows: two blocks and a thin one of 10), nothing on the large head."""
+    cfg = _cfg(B=266, V=20000, H_small=3072, H_large=64, T=2, tau=99.0, d_min=1)
+    wl = synth.Workload(cfg)
+    ora = _oracle(cfg, wl)
+    with GpuGate(cfg, wl.W_small, wl.W_large) as g:
+        out = g.run(wl.h_small, wl.h_large, "run")
+    log = compare(out, ora, cfg.tau)
+    assert log["cells"] == cfg.B * cfg.T and not ora["used"].any()
+
+
 def test_a_step_with_every_sequence_ended_computes_nothing_and_keeps_the_state():
     cfg = _cfg(B=150, V=900, T=6, tau=_mid_tau(900))
     wl = synth.Workload(cfg)
