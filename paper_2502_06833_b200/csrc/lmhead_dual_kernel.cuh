@@ -26,10 +26,10 @@
 // for a two-block unit, three of them): the producer first waits until every stage of the previous
 // head has been consumed.
 //
-// A THIN third block.  A head of 2k + 1 row blocks whose last block has at most 64 rows would pay
+// A THIN third block.  A head of three row blocks whose last block has at most 64 rows would pay
 // a whole single-block unit for them (its own pass of the weights through shared memory, and,
 // because units of different kinds cannot share tiles in L2, a second pass through HBM).  Instead
-// the last two-block unit takes the block along: per stage it also loads the thin block's hidden
+// the two-block unit takes the block along: per stage it also loads the thin block's hidden
 // rows (64 x 64, 8 KiB) and issues, after the MMAs of its two blocks, two more with the operands
 // swapped: A = 128 rows of the weight tile that is in shared memory anyway (rows 0..127, and
 // rows tile_n - 128..tile_n - 1), B = the thin rows, N = thin16 = rows rounded up to 16.  Those
@@ -49,7 +49,8 @@
 // Work split (split_units): the units of a head get CTAs in proportion to their cost (9 : 5 for
 // two blocks : one) and a unit's CTAs take its tiles round-robin (member j takes tiles
 // j, j + g, ...); what is left after the whole rounds is cut into g even pieces, so the members
-// of a unit finish together.  Units of one kind sweep the vocabulary at the same pace whatever
+// of a unit finish together; a share of few tiles is cut into pieces of nearly equal width where
+// that was measured to pay (split_units).  Units of one kind sweep the vocabulary at the same pace whatever
 // their number, so a weight tile fetched for one is an L2 hit for the others; units of different
 // kinds do not (a head with two kinds reads its weights twice: measured).
 #pragma once
